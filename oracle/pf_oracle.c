@@ -1,0 +1,140 @@
+/*
+ * pf_oracle.c -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, fp64 CPU evaluation of the generalized rank-r delta-rule recurrence, token by
+ * token, exactly as the paper defines it.  Nothing here is chunked, blocked, fused or reordered;
+ * there is no W/U compact form and no triangular solve.  Only tests, the smoke check and the
+ * bench's cpu_baseline leg may call it.  It shares no code with the CUDA path.
+ *
+ * What it computes, per (batch b, head h), with S in R^{d_v x d_k}:
+ *
+ *     S_t = S_{t-1} (I - sum_j beta_{t,j} k_{t,j} k_{t,j}^T) + sum_j beta_{t,j} v_{t,j} k_{t,j}^T
+ *     o_t = S_t q_t
+ *
+ * Sources: the (recurrence) / (memory readout) pair of Section 1.1 gives S_t = S_{t-1} <> A_t +
+ * v_t k_t^T and o_t = S_t q_t (readout uses the state AFTER token t's update); the (DeltaNet)
+ * equation of Section 1.3 gives the rank-1 delta rule; Eq. (discretization) of Section 3.1 with
+ * the R=1 Remark generalised to R columns (A_t = K_t diag(beta_t), A~_t = -V_t diag(beta_t),
+ * B_t = -K_t) turns the discrete step  S_{k+1} = S_k + S_k A_k B_k^T + A~_k B_k^T  into the line
+ * above.  All r factors of a token read the SAME old state (diagonal R x R blocks of
+ * Id - M (.) A B^T are the identity, proof of Theorem 3.2), i.e. the "sum" form.
+ *
+ * Every pin that ties this file to something other than itself is in tests/test_oracle_pins.py.
+ *
+ * Layouts (all row-major, host memory):
+ *     q    [B,H,L,d_k]     float   (the exact input values the GPU receives, bf16 or fp32, widened)
+ *     k    [B,H,L,r,d_k]   float
+ *     v    [B,H,L,r,d_v]   float
+ *     beta [B,H,L,r]       float
+ *     S0   [B,H,d_k,d_v]   double or NULL (zeros);  S0[b,h,i,j] = S[j][i]
+ *     O    [B,H,L,d_v]     double
+ *     S_final [B,H,d_k,d_v] double or NULL
+ */
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* One sequence.  S is kept as S[j*d_k + i], j in [0,d_v), i in [0,d_k). */
+static void pf_oracle_one_sequence(const float* q, const float* k, const float* v, const float* beta,
+                                   const double* S0, int L, int d_k, int d_v, int r,
+                                   double* O, double* S_final, double* S, double* p)
+{
+    for (int j = 0; j < d_v; ++j)
+        for (int i = 0; i < d_k; ++i)
+            S[(size_t)j * d_k + i] = S0 ? S0[(size_t)i * d_v + j] : 0.0;
+
+    for (int t = 0; t < L; ++t) {
+        const float* kt = k + (size_t)t * r * d_k;
+        const float* vt = v + (size_t)t * r * d_v;
+        const float* bt = beta + (size_t)t * r;
+
+        /* predictions p_f = S_{t-1} k_{t,f} for every factor f, all from the old state */
+        for (int f = 0; f < r; ++f)
+            for (int j = 0; j < d_v; ++j) {
+                double acc = 0.0;
+                for (int i = 0; i < d_k; ++i)
+                    acc += S[(size_t)j * d_k + i] * (double)kt[(size_t)f * d_k + i];
+                p[(size_t)f * d_v + j] = acc;
+            }
+
+        /* S_t = S_{t-1} + sum_f beta_f (v_f - p_f) k_f^T */
+        for (int f = 0; f < r; ++f) {
+            double b = (double)bt[f];
+            for (int j = 0; j < d_v; ++j) {
+                double e = b * ((double)vt[(size_t)f * d_v + j] - p[(size_t)f * d_v + j]);
+                for (int i = 0; i < d_k; ++i)
+                    S[(size_t)j * d_k + i] += e * (double)kt[(size_t)f * d_k + i];
+            }
+        }
+
+        /* o_t = S_t q_t */
+        const float* qt = q + (size_t)t * d_k;
+        for (int j = 0; j < d_v; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < d_k; ++i)
+                acc += S[(size_t)j * d_k + i] * (double)qt[i];
+            O[(size_t)t * d_v + j] = acc;
+        }
+    }
+
+    if (S_final)
+        for (int j = 0; j < d_v; ++j)
+            for (int i = 0; i < d_k; ++i)
+                S_final[(size_t)i * d_v + j] = S[(size_t)j * d_k + i];
+}
+
+/* Returns 0 on success, -1 on a bad argument, -2 on allocation failure.
+ * num_threads <= 0 means "whatever OpenMP picks"; sequences (b,h) are independent, and that is the
+ * only parallelism used.  *threads_used (may be NULL) receives the thread count actually used. */
+int pf_oracle_deltanet_fwd_f64(const float* q, const float* k, const float* v, const float* beta,
+                               const double* S0, int B, int H, int L, int d_k, int d_v, int r,
+                               double* O, double* S_final, int num_threads, int* threads_used)
+{
+    if (!q || !k || !v || !beta || !O) return -1;
+    if (B < 1 || H < 1 || L < 0 || d_k < 1 || d_v < 1 || r < 1) return -1;
+    const int nseq = B * H;
+    int nt = 1;
+#ifdef _OPENMP
+    nt = num_threads > 0 ? num_threads : omp_get_max_threads();
+    if (nt > nseq) nt = nseq;
+    if (nt < 1) nt = 1;
+#else
+    (void)num_threads;
+#endif
+    if (threads_used) *threads_used = nt;
+    int failed = 0;
+
+#ifdef _OPENMP
+#pragma omp parallel num_threads(nt)
+#endif
+    {
+        double* S = (double*)malloc(sizeof(double) * (size_t)d_v * d_k);
+        double* p = (double*)malloc(sizeof(double) * (size_t)r * d_v);
+        if (!S || !p) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            failed = 1;
+        } else {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+            for (int s = 0; s < nseq; ++s) {
+                pf_oracle_one_sequence(q + (size_t)s * L * d_k,
+                                       k + (size_t)s * L * r * d_k,
+                                       v + (size_t)s * L * r * d_v,
+                                       beta + (size_t)s * L * r,
+                                       S0 ? S0 + (size_t)s * d_k * d_v : NULL,
+                                       L, d_k, d_v, r,
+                                       O + (size_t)s * L * d_v,
+                                       S_final ? S_final + (size_t)s * d_k * d_v : NULL,
+                                       S, p);
+            }
+        }
+        free(S);
+        free(p);
+    }
+    return failed ? -2 : 0;
+}
