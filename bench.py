@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the chunkwise delta-rule forward pass (one "step" = one pass of the whole hot path
+over one batch of the rank-2 workload: B=2, H=16, L=8192, d_k=d_v=128, r=2, chunk=64, bf16 inputs).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+
+Prints ONE JSON line.  `value` is tokens/s (B*L tokens per step, all heads) with inputs resident in
+HBM; `e2e` is the same metric through the C-ABI call with pinned HOST buffers (copies timed);
+`roofline` describes the dominant kernel; `cpu_baseline` is the fp64 oracle timed on this machine's host
+cores.  With --gpus N > 1 (torchrun) every rank runs the same batch on its own GPU (sequences are
+independent: no collective on the data path) and the value is the aggregate.
+`--impl reference` times the fp64 CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import pf_synth  # noqa: E402
+
+METRIC = "tokens/s, rank-2 generalized DeltaNet fwd, L=8192 H=16 d=128"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---- algorithmic work (per token-head unless noted); d_k = d_v = d allowed to differ ----------------
+def alg_bytes_per_token_head(w) -> int:
+    e = 2 if w.dtype == "bf16" else 4
+    return e * (w.d_k + w.r * w.d_k + w.r * w.d_v + w.r) + 4 * w.d_v      # read q,k,v,beta once; write O fp32
+
+
+def flops_per_chunk(w, tri: bool) -> dict:
+    """Chunk-form FLOPs by step; `tri` halves the products the causal masks make half empty."""
+    C, r, dk, dv = w.chunk, w.r, w.d_k, w.d_v
+    n = C * r
+    h = 0.5 if tri else 1.0
+    return {
+        "gram": 2 * n * n * dk * h, "solve": n ** 3 / 3.0, "wu": 2 * n * n * (dk + dv) * h,
+        "attn": 2 * C * n * dk * h, "corr": 2 * n * dk * dv, "out": 2 * C * dk * dv + 2 * C * n * dv * h,
+        "state": 2 * n * dk * dv,
+    }
+
+
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, r[5:9]):
+                if val.strip().lower() == "active":
+                    reasons.add(nm)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def oracle_timed(w, sample_heads: int):
+    """The oracle as it stands on a bounded sample: the first `sample_heads` (b,h) sequences, full L."""
+    import oracle
+    B = 1
+    sub = w.with_(B=B, H=sample_heads)
+    inp = pf_synth.make_inputs(sub)
+    t0 = time.perf_counter()
+    _, _, threads = oracle.deltanet_fwd(inp.q, inp.k, inp.v, inp.beta, inp.S0, return_threads=True)
+    dt = time.perf_counter() - t0
+    token_heads_per_s = sub.token_heads / dt
+    return token_heads_per_s / w.H, threads, dt      # tokens/s for a model with w.H heads
+
+
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    heads = min(w.B * w.H, 16)
+    vals, threads = [], 0
+    for i in range(args.warmup + args.steps):
+        v, threads, dt = oracle_timed(w, heads)
+        if i >= args.warmup:
+            vals.append((v, dt))
+    tok_s = statistics.mean(v for v, _ in vals)
+    ms = statistics.mean(dt for _, dt in vals) * 1e3
+    sample = f"{heads} of {w.B * w.H} (b,h) sequences of {w.name}, all L={w.L} tokens, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tok_s, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_k": w.d_k, "d_v": w.d_v, "r": w.r,
+                   "chunk": w.chunk, "sample": sample},
+        "cpu_baseline": {"value": tok_s, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tok_s, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def kernel_profile(pf, d, w, steps):
+    """Per-kernel device time (ms per launch, averaged) from CUDA events recorded inside the library."""
+    from paper_2504_00492_b200 import binding
+    lib = binding.lib()
+    if not hasattr(lib, "pf_profile_enable"):
+        return {}
+    import ctypes
+    lib.pf_profile_enable(1)
+    acc = {}
+    for _ in range(steps):
+        pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+        torch.cuda.synchronize()
+        n = lib.pf_profile_count()
+        for i in range(n):
+            name = ctypes.create_string_buffer(64)
+            ms = ctypes.c_float(0)
+            lib.pf_profile_read(i, name, 64, ctypes.byref(ms))
+            acc.setdefault(name.value.decode(), []).append(ms.value)
+    lib.pf_profile_enable(0)
+    return {k: statistics.mean(v) for k, v in acc.items()}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(pf_synth.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = pf_synth.CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import paper_2504_00492_b200 as pf
+    peaks, peak_kind = load_peaks()
+
+    host = pf_synth.make_inputs(w, seed=w.seed + 1000 * rank).pin()
+    d = host.to("cuda")
+    O = torch.empty(w.B, w.H, w.L, w.d_v, dtype=torch.float32, device="cuda")
+    Sf = torch.empty(w.B, w.H, w.d_k, w.d_v, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk, O=O, S_final=Sf)
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    launches_per_step = pf.pf_last_launch_count()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record(stream)
+    for i in range(args.steps):
+        step()
+        ev[i + 1].record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else {}
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    if use_dist:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    tokens_per_step = w.tokens * world
+    value = tokens_per_step * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end: pinned host inputs -> device, call, outputs -> pinned host, all timed --------------
+    hO = torch.empty(O.shape, dtype=O.dtype).pin_memory()
+    hS = torch.empty(Sf.shape, dtype=Sf.dtype).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        dd = host.to("cuda", non_blocking=True)
+        o, s = pf.pf_deltanet_fwd(dd.q, dd.k, dd.v, dd.beta, dd.S0, w.chunk, O=O, S_final=Sf)
+        hO.copy_(o, non_blocking=True)
+        hS.copy_(s, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if use_dist:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3)
+    h2d = host.nbytes()
+    d2h = hO.numel() * 4 + hS.numel() * 4
+
+    # ---- per-kernel times and the roofline of the dominant kernel -----------------------------------------
+    prof = kernel_profile(pf, d, w, steps=min(args.steps, 5))
+    G = w.B * w.H * ((w.L + w.chunk - 1) // w.chunk)
+    th = w.token_heads
+    fl_tri = flops_per_chunk(w, tri=True)
+    fl_dense = flops_per_chunk(w, tri=False)
+    ms_step = total_ms / args.steps
+    t_hbm_us = th * alg_bytes_per_token_head(w) / (peaks["hbm_gbs"] * 1e9) * 1e6
+    t_flop_us = G * sum(fl_dense[k] for k in fl_dense if k != "solve") / (peaks["bf16_tflops"] * 1e12) * 1e6
+    path = {"t_hbm_us": t_hbm_us, "t_flop_dense_us": t_flop_us, "frac": max(t_hbm_us, t_flop_us) / (ms_step * 1e3),
+            "peaks": peak_kind, "tflops_dense": G * sum(fl_dense.values()) / (ms_step * 1e-3) / 1e12,
+            "tflops_tri": G * sum(fl_tri.values()) / (ms_step * 1e-3) / 1e12,
+            "hbm_gbs_algorithmic": th * alg_bytes_per_token_head(w) / (ms_step * 1e-3) / 1e9}
+    # which algorithmic steps each kernel covers (triangular-aware FLOPs: the conservative count)
+    kernel_steps = {
+        "simt_gram": ["gram", "attn"], "simt_solve": ["solve"], "simt_wu": ["wu"], "simt_scan": ["corr", "out", "state"],
+        "tc_flow": ["gram", "solve", "wu", "attn"], "tc_scan": ["corr", "out", "state"],
+    }
+    roofline = None
+    if prof:
+        top = max(prof, key=prof.get)
+        steps_of = kernel_steps.get(top, list(fl_tri))
+        fl = G * sum(fl_tri[s] for s in steps_of)
+        achieved = fl / (prof[top] * 1e-3) / 1e12
+        bound = "alu" if top.startswith("simt") else "tensor"
+        # fp32 FFMA peak: 148 SMs x 128 lanes x 2 FLOP x max SM clock
+        peak = 148 * 128 * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12 if bound == "alu" else peaks["bf16_tflops"]
+        roofline = {"bound": bound, "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": None, "ms_per_launch": prof[top], "peaks": peak_kind,
+                    "flops_per_launch": fl, "flop_count": "triangular-aware", "kernel_ms": prof}
+
+    if rank == 0:
+        cpu = None
+        if not args.no_cpu_baseline:
+            heads = min(w.B * w.H, 32)
+            v, threads, dt = oracle_timed(w, heads)
+            cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+                   "sample": f"{heads} of {w.B * w.H} (b,h) sequences of {w.name}, all L={w.L} tokens, {dt:.2f} s wall"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 in / f16 operands / f32 accumulate" if pf.pf_select_impl(
+                w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk) == pf.PF_IMPL_TC else "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_k": w.d_k, "d_v": w.d_v, "r": w.r,
+                       "chunk": w.chunk, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
+                           (host.nbytes() + O.numel() * 4) / 1e6), "parallelism": "replicas" if world > 1 else "1 GPU"},
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+            "token_heads_per_s": value * w.H,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
+            "path_roofline": path, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if use_dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,134 @@
+/*
+ * pf.h -- C ABI of the chunkwise-parallel forward pass of the rank-r generalized delta rule.
+ *
+ * The operation (per batch b and head h, state S in R^{d_v x d_k}):
+ *
+ *     S_t = S_{t-1} (I - sum_j beta_{t,j} k_{t,j} k_{t,j}^T) + sum_j beta_{t,j} v_{t,j} k_{t,j}^T
+ *     o_t = S_t q_t                                   (readout after token t's update)
+ *
+ * This is the associative linear RNN of Section 1.1 (recurrence + memory readout) with the
+ * DeltaNet transition of Section 1.3, generalised to rank-R updates by the drivers of Section 3.1,
+ * Eq. (discretization):  A_t = K_t diag(beta_t),  A~_t = -V_t diag(beta_t),  B_t = -K_t  (the R=1
+ * Remark applied column by column).  All r factors of a token act on the same previous state.
+ *
+ * It is evaluated chunk by chunk in the "Parallel Flows" order of Section 3 (Chunk -> Parallel
+ * Compute -> Scan).  For a chunk of C tokens, rows m = t*r + j, n = C*r, Theorem 3.2 becomes
+ *
+ *     Lm = I + Mstrict (.) (diag(beta) K K^T),      Mstrict[m,m'] = 1(tok(m') < tok(m))
+ *     T' = Lm^{-1} diag(beta),   W = T' K,   Uh = T' V          (compact W/U form of the chunk flow)
+ *     U' = Uh - W S^T,           P = (Q K^T) (.) 1(tok(m) <= t)
+ *     O  = Q S^T + P U',         S <- S + U'^T K                (= S (I - W^T K) + Uh^T K)
+ *
+ * Everything behind these entry points runs in CUDA kernels for sm_100a; there is no CPU path.
+ *
+ * Conventions for every call
+ *   - Tensor pointers are DEVICE pointers owned by the caller, dense row-major in the shapes given;
+ *     the library neither frees nor keeps them.  q/k/v/beta/O must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t (NULL = the default stream).  Work is enqueued; the calls do not
+ *     synchronise.  Unless a workspace is passed through pf_deltanet_fwd_ex, scratch memory is
+ *     taken and returned with stream-ordered allocation on `stream`.
+ *   - O must not alias an input.  S_final may alias S0.
+ *   - Return value: PF_OK (0) or a negative pf_status.  Nothing is launched when an argument check
+ *     fails.  No exceptions, no exit().
+ *   - Supported shapes: d_k, d_v in {64, 128}; r in {1,2,3,4}; chunk in {16, 32, 64}; any L >= 0
+ *     (a ragged last chunk is handled); B, H >= 1.  Anything else returns PF_ERR_UNSUPPORTED --
+ *     there is no slow fallback.
+ */
+#ifndef PF_H_
+#define PF_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pf_status {
+    PF_OK = 0,
+    PF_ERR_INVALID = -1,      /* null pointer, non-positive size, aliasing */
+    PF_ERR_UNSUPPORTED = -2,  /* shape / dtype / impl outside the supported set */
+    PF_ERR_ALIGNMENT = -3,    /* a tensor pointer is not 16-byte aligned */
+    PF_ERR_ARCH = -4,         /* current device is not compute capability 10.x */
+    PF_ERR_CUDA = -5,         /* a CUDA runtime call failed; see pf_last_error_string() */
+    PF_ERR_WORKSPACE = -6,    /* caller workspace too small or misaligned */
+    PF_ERR_TIMEOUT = -7       /* a bounded device-side wait expired (reported via status word) */
+} pf_status;
+
+enum { PF_DTYPE_BF16 = 0, PF_DTYPE_F32 = 1 };
+
+/* Which kernels evaluate the chunk form.
+ *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.
+ *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
+ *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.   */
+enum { PF_IMPL_AUTO = 0, PF_IMPL_SIMT = 1, PF_IMPL_TC = 2 };
+
+/*
+ * pf_deltanet_fwd -- the central call: bf16 inputs, fp32 accumulation, fp32 outputs.
+ *   q    [B,H,L,d_k]     bf16
+ *   k    [B,H,L,r,d_k]   bf16     row (t,j) contiguous
+ *   v    [B,H,L,r,d_v]   bf16
+ *   beta [B,H,L,r]       bf16
+ *   S0   [B,H,d_k,d_v]   fp32 or NULL (zero state);  S0[b,h,i,j] = S[j][i]
+ *   O    [B,H,L,d_v]     fp32     (written)
+ *   S_final [B,H,d_k,d_v] fp32 or NULL (not wanted)   (written)
+ * Defined by: recurrence/readout of Section 1.1, delta rule of Section 1.3, rank-R drivers of
+ * Section 3.1, evaluated per chunk through Theorem 3.2 and carried across chunks (Section 3).
+ */
+int pf_deltanet_fwd(const void* q, const void* k, const void* v, const void* beta, const float* S0,
+                    int B, int H, int L, int d_k, int d_v, int r, int chunk,
+                    float* O, float* S_final, void* stream);
+
+/* Same operation with fp32 q, k, v, beta (all arithmetic fp32 FFMA).  Same passages. */
+int pf_deltanet_fwd_f32(const float* q, const float* k, const float* v, const float* beta,
+                        const float* S0, int B, int H, int L, int d_k, int d_v, int r, int chunk,
+                        float* O, float* S_final, void* stream);
+
+typedef struct pf_params {
+    const void* q;            /* as in pf_deltanet_fwd, element type given by in_dtype */
+    const void* k;
+    const void* v;
+    const void* beta;
+    const float* S0;
+    int B, H, L, d_k, d_v, r, chunk;
+    float* O;
+    float* S_final;
+    int in_dtype;             /* PF_DTYPE_BF16 or PF_DTYPE_F32 */
+    int impl;                 /* PF_IMPL_* */
+    void* workspace;          /* device scratch of >= pf_workspace_bytes(...) bytes, 256-byte aligned,
+                                 or NULL: stream-ordered allocation inside the call */
+    size_t workspace_bytes;
+    void* stream;
+} pf_params;
+
+/* Same operation with explicit options.  The workspace holds per-chunk intermediates (T', W, Uh, P
+ * of Theorem 3.2 in the forms the selected kernels exchange); its content after the call is
+ * unspecified.  Same passages as pf_deltanet_fwd. */
+int pf_deltanet_fwd_ex(const pf_params* p);
+
+/* Bytes of scratch pf_deltanet_fwd_ex needs for this problem with this in_dtype/impl (0 on an
+ * unsupported combination).  Host-only arithmetic; no CUDA call. */
+size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
+
+/* Which PF_IMPL_* pf_deltanet_fwd_ex would run for this problem (negative pf_status if none). */
+int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
+
+/* Number of kernels the last successful call on this host thread enqueued. */
+int pf_last_launch_count(void);
+
+/* Optional per-kernel timing for benchmarks.  While enabled, each kernel of a forward call is
+ * bracketed by CUDA events on the call's stream.  After the call, pf_profile_count() gives the number
+ * of kernels and pf_profile_read(i, ...) waits for kernel i to finish and returns its name and device
+ * time in milliseconds.  Process-wide, not thread-safe; leave it off in production. */
+void pf_profile_enable(int on);
+int pf_profile_count(void);
+int pf_profile_read(int idx, char* name, int name_cap, float* ms);
+
+const char* pf_status_string(int status);
+/* Text of the last CUDA error seen by this host thread inside the library ("" if none). */
+const char* pf_last_error_string(void);
+int pf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PF_H_ */

@@ -1,0 +1,200 @@
+"""ctypes binding of libpf.so: argument marshalling only -- every step runs in the CUDA kernels.
+
+The function names mirror the C ABI in include/pf.h.  Tensors are torch CUDA tensors (torch is
+used for device memory and streams only).  If the library is missing or cannot be loaded the
+import of this module fails loudly; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libpf.so")
+
+PF_DTYPE_BF16, PF_DTYPE_F32 = 0, 1
+PF_IMPL_AUTO, PF_IMPL_SIMT, PF_IMPL_TC = 0, 1, 2
+IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC}
+
+# every symbol include/pf.h declares
+EXPORTS = [
+    "pf_deltanet_fwd", "pf_deltanet_fwd_f32", "pf_deltanet_fwd_ex", "pf_workspace_bytes", "pf_select_impl",
+    "pf_last_launch_count", "pf_status_string", "pf_last_error_string", "pf_version",
+    "pf_profile_enable", "pf_profile_count", "pf_profile_read",
+]
+
+
+class PfParams(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("beta", ctypes.c_void_p),
+        ("S0", ctypes.c_void_p),
+        ("B", ctypes.c_int), ("H", ctypes.c_int), ("L", ctypes.c_int), ("d_k", ctypes.c_int),
+        ("d_v", ctypes.c_int), ("r", ctypes.c_int), ("chunk", ctypes.c_int),
+        ("O", ctypes.c_void_p), ("S_final", ctypes.c_void_p),
+        ("in_dtype", ctypes.c_int), ("impl", ctypes.c_int),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
+class PfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().pf_status_string(status).decode()
+        detail = lib().pf_last_error_string().decode()
+        super().__init__(f"{where}: {msg} ({status})" + (f": {detail}" if status == -5 and detail else ""))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2504_00492_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        L.pf_deltanet_fwd.restype = ci
+        L.pf_deltanet_fwd.argtypes = [vp] * 5 + [ci] * 7 + [vp, vp, vp]
+        L.pf_deltanet_fwd_f32.restype = ci
+        L.pf_deltanet_fwd_f32.argtypes = [vp] * 5 + [ci] * 7 + [vp, vp, vp]
+        L.pf_deltanet_fwd_ex.restype = ci
+        L.pf_deltanet_fwd_ex.argtypes = [ctypes.POINTER(PfParams)]
+        L.pf_workspace_bytes.restype = ctypes.c_size_t
+        L.pf_workspace_bytes.argtypes = [ci] * 9
+        L.pf_select_impl.restype = ci
+        L.pf_select_impl.argtypes = [ci] * 9
+        L.pf_last_launch_count.restype = ci
+        L.pf_last_launch_count.argtypes = []
+        L.pf_status_string.restype = ctypes.c_char_p
+        L.pf_status_string.argtypes = [ci]
+        L.pf_last_error_string.restype = ctypes.c_char_p
+        L.pf_last_error_string.argtypes = []
+        L.pf_version.restype = ci
+        L.pf_version.argtypes = []
+        L.pf_profile_enable.restype = None
+        L.pf_profile_enable.argtypes = [ci]
+        L.pf_profile_count.restype = ci
+        L.pf_profile_count.argtypes = []
+        L.pf_profile_read.restype = ci
+        L.pf_profile_read.argtypes = [ci, ctypes.c_char_p, ci, ctypes.POINTER(ctypes.c_float)]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _check_inputs(q, k, v, beta, S0, dtype) -> Tuple[int, int, int, int, int, int]:
+    if k.dim() != 5 or q.dim() != 4 or v.dim() != 5 or beta.dim() != 4:
+        raise ValueError("expected q [B,H,L,d_k], k [B,H,L,r,d_k], v [B,H,L,r,d_v], beta [B,H,L,r]")
+    B, H, L, r, d_k = k.shape
+    d_v = v.shape[-1]
+    if tuple(q.shape) != (B, H, L, d_k) or tuple(v.shape) != (B, H, L, r, d_v) or tuple(beta.shape) != (B, H, L, r):
+        raise ValueError("inconsistent input shapes")
+    for name, t in (("q", q), ("k", k), ("v", v), ("beta", beta)):
+        if t.dtype != dtype:
+            raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+        if not t.is_cuda:
+            raise ValueError(f"{name} must be a CUDA tensor")
+        if not t.is_contiguous():
+            raise ValueError(f"{name} must be contiguous")
+    if S0 is not None:
+        if S0.dtype != torch.float32 or tuple(S0.shape) != (B, H, d_k, d_v) or not S0.is_cuda or not S0.is_contiguous():
+            raise ValueError("S0 must be a contiguous fp32 CUDA tensor [B,H,d_k,d_v]")
+    return B, H, L, d_k, d_v, r
+
+
+def _outputs(q, B, H, L, d_k, d_v, O, S_final, want_state):
+    if O is None:
+        O = torch.empty(B, H, L, d_v, dtype=torch.float32, device=q.device)
+    if S_final is None and want_state:
+        S_final = torch.empty(B, H, d_k, d_v, dtype=torch.float32, device=q.device)
+    return O, S_final
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def pf_deltanet_fwd(q, k, v, beta, S0, chunk: int, O=None, S_final=None, stream=None, want_state: bool = True):
+    """bf16 q/k/v/beta -> (O fp32 [B,H,L,d_v], S_final fp32 [B,H,d_k,d_v] or None)."""
+    B, H, L, d_k, d_v, r = _check_inputs(q, k, v, beta, S0, torch.bfloat16)
+    O, S_final = _outputs(q, B, H, L, d_k, d_v, O, S_final, want_state)
+    with torch.cuda.device(q.device):
+        st = lib().pf_deltanet_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(S0), B, H, L, d_k, d_v, r, chunk,
+                                   _ptr(O), _ptr(S_final), _stream(stream))
+    if st != 0:
+        raise PfError(st, "pf_deltanet_fwd")
+    return O, S_final
+
+
+def pf_deltanet_fwd_f32(q, k, v, beta, S0, chunk: int, O=None, S_final=None, stream=None, want_state: bool = True):
+    """fp32 q/k/v/beta -> (O, S_final), all arithmetic fp32."""
+    B, H, L, d_k, d_v, r = _check_inputs(q, k, v, beta, S0, torch.float32)
+    O, S_final = _outputs(q, B, H, L, d_k, d_v, O, S_final, want_state)
+    with torch.cuda.device(q.device):
+        st = lib().pf_deltanet_fwd_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(S0), B, H, L, d_k, d_v, r, chunk,
+                                       _ptr(O), _ptr(S_final), _stream(stream))
+    if st != 0:
+        raise PfError(st, "pf_deltanet_fwd_f32")
+    return O, S_final
+
+
+def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Optional[torch.Tensor] = None,
+                       O=None, S_final=None, stream=None, want_state: bool = True):
+    """Same operation with an explicit implementation and (optionally) a caller-owned workspace
+    (a uint8 CUDA tensor of at least pf_workspace_bytes(...) bytes)."""
+    dtype = q.dtype
+    if dtype not in (torch.bfloat16, torch.float32):
+        raise TypeError("q/k/v/beta must be bf16 or fp32")
+    B, H, L, d_k, d_v, r = _check_inputs(q, k, v, beta, S0, dtype)
+    O, S_final = _outputs(q, B, H, L, d_k, d_v, O, S_final, want_state)
+    p = PfParams()
+    p.q, p.k, p.v, p.beta, p.S0 = _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(S0)
+    p.B, p.H, p.L, p.d_k, p.d_v, p.r, p.chunk = B, H, L, d_k, d_v, r, chunk
+    p.O, p.S_final = _ptr(O), _ptr(S_final)
+    p.in_dtype = PF_DTYPE_F32 if dtype == torch.float32 else PF_DTYPE_BF16
+    p.impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
+    if workspace is not None:
+        p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    p.stream = _stream(stream)
+    with torch.cuda.device(q.device):
+        st = lib().pf_deltanet_fwd_ex(ctypes.byref(p))
+    if st != 0:
+        raise PfError(st, "pf_deltanet_fwd_ex")
+    return O, S_final
+
+
+def pf_workspace_bytes(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
+    impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
+    return int(lib().pf_workspace_bytes(B, H, L, d_k, d_v, r, chunk, in_dtype, impl))
+
+
+def pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
+    impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
+    return int(lib().pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype, impl))
+
+
+def pf_last_launch_count() -> int:
+    return int(lib().pf_last_launch_count())
+
+
+def pf_status_string(status: int) -> str:
+    return lib().pf_status_string(status).decode()
+
+
+def pf_last_error_string() -> str:
+    return lib().pf_last_error_string().decode()
+
+
+def pf_version() -> int:
+    return int(lib().pf_version())

@@ -1,0 +1,211 @@
+// extern "C" entry points: argument checks, implementation choice, scratch memory, dispatch.
+#include <stdio.h>
+#include <string.h>
+
+#include "pf_common.cuh"
+
+namespace pf {
+
+static thread_local char g_err[512] = "";
+static thread_local int g_launches = 0;
+static thread_local int g_launch_accum = 0;
+
+int record_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_err, sizeof(g_err), "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
+    return PF_ERR_CUDA;
+}
+
+void count_launch(int n) { g_launch_accum += n; }
+
+// ---- optional per-kernel timing ---------------------------------------------------------------
+struct ProfEntry {
+    char name[48];
+    cudaEvent_t e0, e1;
+};
+static bool g_prof_on = false;
+static ProfEntry g_prof[64];
+static int g_prof_n = 0;       // entries of the current call
+static int g_prof_made = 0;    // events created so far
+
+void prof_begin(const char* name, cudaStream_t stream) {
+    if (!g_prof_on || g_prof_n >= 64) return;
+    ProfEntry& e = g_prof[g_prof_n];
+    if (g_prof_n >= g_prof_made) {
+        if (cudaEventCreate(&e.e0) != cudaSuccess || cudaEventCreate(&e.e1) != cudaSuccess) return;
+        g_prof_made = g_prof_n + 1;
+    }
+    snprintf(e.name, sizeof(e.name), "%s", name);
+    cudaEventRecord(e.e0, stream);
+}
+
+void prof_end(cudaStream_t stream) {
+    if (!g_prof_on || g_prof_n >= 64 || g_prof_n >= g_prof_made) return;
+    cudaEventRecord(g_prof[g_prof_n].e1, stream);
+    ++g_prof_n;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+int check_shape(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
+    if (B < 1 || H < 1 || L < 0) return PF_ERR_INVALID;
+    if (!(d_k == 64 || d_k == 128) || !(d_v == 64 || d_v == 128)) return PF_ERR_UNSUPPORTED;
+    if (r < 1 || r > 4) return PF_ERR_UNSUPPORTED;
+    if (!(chunk == 16 || chunk == 32 || chunk == 64)) return PF_ERR_UNSUPPORTED;
+    return PF_OK;
+}
+
+Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype) {
+    Problem p{};
+    p.B = B; p.H = H; p.L = L; p.d_k = d_k; p.d_v = d_v; p.r = r; p.chunk = chunk;
+    p.in_dtype = in_dtype;
+    return p;
+}
+
+int select_impl(const Problem& p, int impl) {
+    if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
+    switch (impl) {
+        case PF_IMPL_SIMT: return PF_IMPL_SIMT;
+        case PF_IMPL_TC: return tc_supported(p) ? (int)PF_IMPL_TC : (int)PF_ERR_UNSUPPORTED;
+        case PF_IMPL_AUTO: return tc_supported(p) ? PF_IMPL_TC : PF_IMPL_SIMT;
+        default: return PF_ERR_UNSUPPORTED;
+    }
+}
+
+bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
+    if (!a || !b || an == 0 || bn == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bn && b0 < a0 + an;
+}
+
+int forward(const pf_params* a) {
+    if (!a) return PF_ERR_INVALID;
+    int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
+    if (st != PF_OK) return st;
+    Problem p = as_problem(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk, a->in_dtype);
+    const int impl = select_impl(p, a->impl);
+    if (impl < 0) return impl;
+    if (a->L > 0 && (!a->q || !a->k || !a->v || !a->beta || !a->O)) return PF_ERR_INVALID;
+    if (!aligned16(a->q) || !aligned16(a->k) || !aligned16(a->v) || !aligned16(a->beta) || !aligned16(a->O) ||
+        !aligned16(a->S0) || !aligned16(a->S_final))
+        return PF_ERR_ALIGNMENT;
+    const size_t es = a->in_dtype == PF_DTYPE_F32 ? 4 : 2;
+    const size_t th = (size_t)a->B * a->H * a->L;
+    const size_t o_bytes = th * a->d_v * 4;
+    if (overlaps(a->O, o_bytes, a->q, th * a->d_k * es) || overlaps(a->O, o_bytes, a->k, th * a->r * a->d_k * es) ||
+        overlaps(a->O, o_bytes, a->v, th * a->r * a->d_v * es) || overlaps(a->O, o_bytes, a->beta, th * a->r * es))
+        return PF_ERR_INVALID;
+
+    int dev = 0;
+    PF_CUDA_TRY(cudaGetDevice(&dev));
+    int major = 0;
+    PF_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) return PF_ERR_ARCH;
+
+    p.q = a->q; p.k = a->k; p.v = a->v; p.beta = a->beta; p.S0 = a->S0;
+    p.O = a->O; p.S_final = a->S_final;
+    p.stream = (cudaStream_t)a->stream;
+
+    const size_t need = impl == PF_IMPL_TC ? tc_workspace_bytes(p) : simt_workspace_bytes(p);
+    void* ws = a->workspace;
+    bool own = false;
+    if (ws) {
+        if (a->workspace_bytes < need || ((uintptr_t)ws & 255u)) return PF_ERR_WORKSPACE;
+    } else if (need > 0) {
+        PF_CUDA_TRY(cudaMallocAsync(&ws, need, p.stream));
+        own = true;
+    }
+    g_launch_accum = 0;
+    g_prof_n = 0;
+    st = impl == PF_IMPL_TC ? tc_forward(p, ws) : simt_forward(p, ws);
+    if (own) {
+        cudaError_t e = cudaFreeAsync(ws, p.stream);
+        if (e != cudaSuccess && st == PF_OK) st = record_cuda_error(e, "cudaFreeAsync");
+    }
+    if (st == PF_OK) g_launches = g_launch_accum;
+    return st;
+}
+
+}  // namespace
+}  // namespace pf
+
+extern "C" {
+
+int pf_deltanet_fwd_ex(const pf_params* p) { return pf::forward(p); }
+
+int pf_deltanet_fwd(const void* q, const void* k, const void* v, const void* beta, const float* S0, int B, int H,
+                    int L, int d_k, int d_v, int r, int chunk, float* O, float* S_final, void* stream) {
+    pf_params a;
+    memset(&a, 0, sizeof(a));
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.S0 = S0;
+    a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
+    a.O = O; a.S_final = S_final;
+    a.in_dtype = PF_DTYPE_BF16;
+    a.impl = PF_IMPL_AUTO;
+    a.stream = stream;
+    return pf::forward(&a);
+}
+
+int pf_deltanet_fwd_f32(const float* q, const float* k, const float* v, const float* beta, const float* S0, int B,
+                        int H, int L, int d_k, int d_v, int r, int chunk, float* O, float* S_final, void* stream) {
+    pf_params a;
+    memset(&a, 0, sizeof(a));
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.S0 = S0;
+    a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
+    a.O = O; a.S_final = S_final;
+    a.in_dtype = PF_DTYPE_F32;
+    a.impl = PF_IMPL_AUTO;
+    a.stream = stream;
+    return pf::forward(&a);
+}
+
+size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
+    if (pf::check_shape(B, H, L, d_k, d_v, r, chunk) != PF_OK) return 0;
+    pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
+    const int sel = pf::select_impl(p, impl);
+    if (sel < 0) return 0;
+    return sel == PF_IMPL_TC ? pf::tc_workspace_bytes(p) : pf::simt_workspace_bytes(p);
+}
+
+int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
+    const int st = pf::check_shape(B, H, L, d_k, d_v, r, chunk);
+    if (st != PF_OK) return st;
+    return pf::select_impl(pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype), impl);
+}
+
+int pf_last_launch_count(void) { return pf::g_launches; }
+
+void pf_profile_enable(int on) { pf::g_prof_on = on != 0; }
+
+int pf_profile_count(void) { return pf::g_prof_n; }
+
+int pf_profile_read(int idx, char* name, int name_cap, float* ms) {
+    if (idx < 0 || idx >= pf::g_prof_n || !ms) return PF_ERR_INVALID;
+    pf::ProfEntry& e = pf::g_prof[idx];
+    cudaError_t err = cudaEventSynchronize(e.e1);
+    if (err == cudaSuccess) err = cudaEventElapsedTime(ms, e.e0, e.e1);
+    if (err != cudaSuccess) return pf::record_cuda_error(err, "pf_profile_read");
+    if (name && name_cap > 0) snprintf(name, (size_t)name_cap, "%s", e.name);
+    return PF_OK;
+}
+
+const char* pf_status_string(int s) {
+    switch (s) {
+        case PF_OK: return "ok";
+        case PF_ERR_INVALID: return "invalid argument";
+        case PF_ERR_UNSUPPORTED: return "unsupported shape, dtype or implementation";
+        case PF_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case PF_ERR_ARCH: return "device is not compute capability 10.x";
+        case PF_ERR_CUDA: return "CUDA error";
+        case PF_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case PF_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* pf_last_error_string(void) { return pf::g_err; }
+
+int pf_version(void) { return 100; }
+
+}  // extern "C"

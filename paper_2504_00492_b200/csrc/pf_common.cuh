@@ -1,0 +1,58 @@
+// Shared host/device definitions of the pf library (internal; the public ABI is include/pf.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pf.h"
+
+namespace pf {
+
+// One forward problem as the launchers see it.
+struct Problem {
+    const void* q;
+    const void* k;
+    const void* v;
+    const void* beta;
+    const float* S0;
+    int B, H, L, d_k, d_v, r, chunk;
+    float* O;
+    float* S_final;
+    int in_dtype;
+    cudaStream_t stream;
+
+    __host__ __device__ int n() const { return chunk * r; }            // rows per chunk
+    __host__ __device__ int chunks_per_seq() const { return (L + chunk - 1) / chunk; }
+    __host__ __device__ long long total_chunks() const { return (long long)B * H * chunks_per_seq(); }
+};
+
+// Records a CUDA error for pf_last_error_string(); returns PF_ERR_CUDA.
+int record_cuda_error(cudaError_t e, const char* where);
+void count_launch(int n = 1);
+
+#define PF_CUDA_TRY(expr)                                             \
+    do {                                                              \
+        cudaError_t _e = (expr);                                      \
+        if (_e != cudaSuccess) return ::pf::record_cuda_error(_e, #expr); \
+    } while (0)
+
+// Optional per-kernel timing (pf_profile_*): when enabled, prof_begin/prof_end bracket a launch
+// with CUDA events on its stream; otherwise they do nothing.
+void prof_begin(const char* name, cudaStream_t stream);
+void prof_end(cudaStream_t stream);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// fp32 SIMT path (pf_simt.cu)
+size_t simt_workspace_bytes(const Problem& p);
+int simt_forward(const Problem& p, void* workspace);
+
+// tcgen05 path (pf_tc.cu)
+bool tc_supported(const Problem& p);
+size_t tc_workspace_bytes(const Problem& p);
+int tc_forward(const Problem& p, void* workspace);
+
+}  // namespace pf

@@ -1,0 +1,166 @@
+"""GPU parity: the CUDA path against the fp64 oracle on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import pf_synth
+from pf_synth import Workload
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    # several chunks + ragged tail, d_k != d_v, every r, every chunk size
+    Workload("s_r1", B=2, H=2, L=200, d_k=64, d_v=128, r=1, chunk=64, s0_std=0.1, seed=11),
+    Workload("s_r2", B=1, H=3, L=150, d_k=128, d_v=64, r=2, chunk=32, s0_std=0.1, seed=12),
+    Workload("s_r3", B=2, H=1, L=97, d_k=64, d_v=64, r=3, chunk=16, beta_scale=2.0, seed=13),
+    Workload("s_r4", B=1, H=2, L=260, d_k=128, d_v=128, r=4, chunk=64, beta_scale=2.0, s0_std=0.1, seed=14),
+    Workload("s_one_token", B=1, H=1, L=1, d_k=64, d_v=64, r=2, chunk=64, s0_std=0.1, seed=15),
+    Workload("s_exact_chunks", B=1, H=2, L=128, d_k=64, d_v=64, r=1, chunk=64, seed=16),
+]
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_cases_simt(w, dtype):
+    util.check_parity(w.with_(dtype=dtype), impl="simt")
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+def test_small_cases_default_impl(w):
+    util.check_parity(w, impl="auto")
+
+
+def test_config0_fp32():
+    import paper_2504_00492_b200 as pf
+    w = pf_synth.CONFIGS["c0"]
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd_f32(d.q, d.k, d.v, d.beta, None, w.chunk)
+    O_ref, Sf_ref = util.run_oracle(inp)
+    assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_F32
+    assert util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_F32
+    assert pf.pf_last_launch_count() > 0
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c3_chunk32"])
+def test_full_configs(name):
+    """Full benchmark sizes through the central call, in the configuration bench.py times."""
+    import paper_2504_00492_b200 as pf
+    w = pf_synth.CONFIGS[name]
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    torch.cuda.synchronize()
+    O_ref, Sf_ref = util.run_oracle(inp)
+    eo, es = util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_config4_long_context_sampled_heads():
+    """c4 at full size on the GPU; the oracle recomputes a sample of whole heads (heads are
+    independent sequences, so each sampled head is checked over all 65536 tokens)."""
+    import paper_2504_00492_b200 as pf
+    w = pf_synth.CONFIGS["c4"]
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    torch.cuda.synchronize()
+    heads = [0, 7, 18, 31]
+    sub = pf_synth.Inputs(inp.q[:, heads].contiguous(), inp.k[:, heads].contiguous(), inp.v[:, heads].contiguous(),
+                          inp.beta[:, heads].contiguous(), inp.S0[:, heads].contiguous())
+    O_ref, Sf_ref = util.run_oracle(sub)
+    eo = util.max_rel(O[:, heads].cpu().numpy(), O_ref)
+    es = util.max_rel(Sf[:, heads].cpu().numpy(), Sf_ref)
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+    assert torch.isfinite(O).all() and torch.isfinite(Sf).all()
+
+
+# --- properties that hold at any size -------------------------------------------------------------
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+def test_split_invariance_and_state_carry(impl):
+    """Proposition 2.1: running [0,L1) then [L1,L) with S_final -> S0 equals one call."""
+    import paper_2504_00492_b200 as pf
+    w = Workload("split", B=1, H=2, L=256, d_k=64, d_v=128, r=2, chunk=32, s0_std=0.1, seed=21)
+    d = pf_synth.make_inputs(w).to("cuda")
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl)
+    L1 = 96
+    O1, S1 = pf.pf_deltanet_fwd_ex(d.q[:, :, :L1].contiguous(), d.k[:, :, :L1].contiguous(),
+                                   d.v[:, :, :L1].contiguous(), d.beta[:, :, :L1].contiguous(), d.S0, w.chunk, impl=impl)
+    O2, S2 = pf.pf_deltanet_fwd_ex(d.q[:, :, L1:].contiguous(), d.k[:, :, L1:].contiguous(),
+                                   d.v[:, :, L1:].contiguous(), d.beta[:, :, L1:].contiguous(), S1, w.chunk, impl=impl)
+    tol = 2e-3
+    assert util.max_rel(torch.cat([O1, O2], 2).cpu().numpy(), O.cpu().numpy()) <= tol
+    assert util.max_rel(S2.cpu().numpy(), Sf.cpu().numpy()) <= tol
+
+
+def test_chunk_size_invariance_fp32():
+    import paper_2504_00492_b200 as pf
+    w = Workload("chunkinv", B=1, H=2, L=192, d_k=64, d_v=64, r=2, chunk=64, dtype="f32", s0_std=0.1, seed=22)
+    d = pf_synth.make_inputs(w).to("cuda")
+    outs = [pf.pf_deltanet_fwd_f32(d.q, d.k, d.v, d.beta, d.S0, c) for c in (16, 32, 64)]
+    for O, Sf in outs[1:]:
+        assert util.max_rel(O.cpu().numpy(), outs[0][0].cpu().numpy()) <= 2e-5
+        assert util.max_rel(Sf.cpu().numpy(), outs[0][1].cpu().numpy()) <= 2e-5
+
+
+def test_beta_zero_and_empty_sequence():
+    import paper_2504_00492_b200 as pf
+    w = Workload("bz", B=1, H=2, L=70, d_k=64, d_v=64, r=2, chunk=32, s0_std=0.1, seed=23)
+    d = pf_synth.make_inputs(w).to("cuda")
+    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, torch.zeros_like(d.beta), d.S0, w.chunk)
+    assert torch.equal(Sf, d.S0)
+    ref = torch.einsum("bhij,bhti->bhtj", d.S0.double(), d.q.double())
+    assert util.max_rel(O.cpu().numpy(), ref.cpu().numpy()) <= util.TOL_BF16
+    # L = 0: nothing to do but hand the state through
+    e = lambda *s: torch.empty(*s, dtype=torch.bfloat16, device="cuda")
+    O0, S0f = pf.pf_deltanet_fwd(e(1, 2, 0, 64), e(1, 2, 0, 2, 64), e(1, 2, 0, 2, 64), e(1, 2, 0, 2), d.S0, 32)
+    assert O0.shape == (1, 2, 0, 64) and torch.equal(S0f, d.S0)
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+def test_deterministic_and_workspace_bounds(impl):
+    """No atomics anywhere: two runs are bitwise equal; a caller workspace is never overrun."""
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    w = Workload("det", B=2, H=2, L=130, d_k=64, d_v=64, r=3, chunk=32, s0_std=0.1, seed=24)
+    d = pf_synth.make_inputs(w).to("cuda")
+    need = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, impl)
+    guard = 4096
+    buf = torch.full((need + 2 * guard + 256,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = (-buf.data_ptr() - guard) % 256 + guard
+    ws = buf[off:off + need]
+    assert ws.data_ptr() % 256 == 0
+    O1, S1 = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws)
+    O2, S2 = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl)
+    torch.cuda.synchronize()
+    assert torch.equal(O1, O2) and torch.equal(S1, S2)
+    assert bool((buf[:off] == 0x5A).all()) and bool((buf[off + need:] == 0x5A).all())
+    with pytest.raises(pf.PfError) as ei:
+        pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[: max(need - 256, 0)])
+    assert ei.value.status == -6
+
+
+def test_argument_errors_launch_nothing():
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    w = Workload("err", B=1, H=1, L=64, d_k=64, d_v=64, r=1, chunk=64, seed=25)
+    d = pf_synth.make_inputs(w).to("cuda")
+    O = torch.zeros(1, 1, 64, 64, device="cuda")
+    lib = binding.lib()
+    st = torch.cuda.current_stream().cuda_stream
+    # misaligned q
+    rc = lib.pf_deltanet_fwd(d.q.data_ptr() + 2, d.k.data_ptr(), d.v.data_ptr(), d.beta.data_ptr(), None,
+                             1, 1, 64, 64, 64, 1, 64, O.data_ptr(), None, st)
+    assert rc == -3
+    # null k
+    rc = lib.pf_deltanet_fwd(d.q.data_ptr(), None, d.v.data_ptr(), d.beta.data_ptr(), None,
+                             1, 1, 64, 64, 64, 1, 64, O.data_ptr(), None, st)
+    assert rc == -1
+    # O aliasing v
+    rc = lib.pf_deltanet_fwd(d.q.data_ptr(), d.k.data_ptr(), d.v.data_ptr(), d.beta.data_ptr(), None,
+                             1, 1, 64, 64, 64, 1, 64, d.v.data_ptr(), None, st)
+    assert rc == -1
+    torch.cuda.synchronize()
+    assert float(O.abs().sum()) == 0.0

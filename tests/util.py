@@ -1,0 +1,47 @@
+"""Helpers shared by the GPU parity tests."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import pf_synth
+
+TOL_BF16 = 2e-3   # bf16 inputs: max|gpu - ref| / max|ref| per tensor
+TOL_F32 = 1e-5    # fp32 path
+
+
+def max_rel(x, ref) -> float:
+    """max_i |x_i - ref_i| / max_i |ref_i| over the whole tensor."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    den = np.abs(ref).max() if ref.size else 0.0
+    if ref.size == 0:
+        return 0.0
+    if den == 0.0:
+        return float(np.abs(x - ref).max())
+    return float(np.abs(x - ref).max() / den)
+
+
+def run_gpu(w: pf_synth.Workload, inp: pf_synth.Inputs, impl="auto", chunk=None, workspace=None):
+    import paper_2504_00492_b200 as pf
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, chunk or w.chunk, impl=impl, workspace=workspace)
+    torch.cuda.synchronize()
+    return O.cpu().numpy(), Sf.cpu().numpy()
+
+
+def run_oracle(inp: pf_synth.Inputs):
+    return oracle.deltanet_fwd(inp.q, inp.k, inp.v, inp.beta, inp.S0)
+
+
+def check_parity(w: pf_synth.Workload, impl="auto", tol=None, inp=None):
+    inp = inp or pf_synth.make_inputs(w)
+    tol = tol if tol is not None else (TOL_F32 if w.dtype == "f32" else TOL_BF16)
+    O, Sf = run_gpu(w, inp, impl=impl)
+    O_ref, Sf_ref = run_oracle(inp)
+    assert np.isfinite(O).all() and np.isfinite(Sf).all()
+    eo, es = max_rel(O, O_ref), max_rel(Sf, Sf_ref)
+    assert eo <= tol, f"{w.name}: O error {eo:.3e} > {tol}"
+    assert es <= tol, f"{w.name}: S_final error {es:.3e} > {tol}"
+    return eo, es
