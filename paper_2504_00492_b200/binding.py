@@ -23,7 +23,7 @@ IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC}
 EXPORTS = [
     "pf_deltanet_fwd", "pf_deltanet_fwd_f32", "pf_deltanet_fwd_ex", "pf_workspace_bytes", "pf_select_impl",
     "pf_last_launch_count", "pf_status_string", "pf_last_error_string", "pf_version",
-    "pf_profile_enable", "pf_profile_count", "pf_profile_read",
+    "pf_profile_enable", "pf_profile_count", "pf_profile_read", "pf_tc_selftest",
 ]
 
 
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.pf_profile_count.argtypes = []
         L.pf_profile_read.restype = ci
         L.pf_profile_read.argtypes = [ci, ctypes.c_char_p, ci, ctypes.POINTER(ctypes.c_float)]
+        L.pf_tc_selftest.restype = ci
+        L.pf_tc_selftest.argtypes = [ci, vp, vp, vp, ci, vp]
         _lib = L
     return _lib
 
