@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_PKG, "libpf.so")
 
 PF_DTYPE_BF16, PF_DTYPE_F32 = 0, 1
 PF_IMPL_AUTO, PF_IMPL_SIMT, PF_IMPL_TC = 0, 1, 2
-IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC}
+PF_IMPL_TC_REFFLOW = 3
+IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC, "tc_refflow": PF_IMPL_TC_REFFLOW}
 
 # every symbol include/pf.h declares
 EXPORTS = [

@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include "pf_common.cuh"
+#include "pf_tc.cuh"
 
 namespace pf {
 
@@ -69,8 +70,15 @@ int select_impl(const Problem& p, int impl) {
         case PF_IMPL_SIMT: return PF_IMPL_SIMT;
         case PF_IMPL_TC: return tc_supported(p) ? (int)PF_IMPL_TC : (int)PF_ERR_UNSUPPORTED;
         case PF_IMPL_AUTO: return tc_supported(p) ? PF_IMPL_TC : PF_IMPL_SIMT;
+        case PF_IMPL_TC_REFFLOW: return tc_scan_supported(p) ? (int)PF_IMPL_TC_REFFLOW : (int)PF_ERR_UNSUPPORTED;
         default: return PF_ERR_UNSUPPORTED;
     }
+}
+
+size_t workspace_need(const Problem& p, int impl) {
+    if (impl == PF_IMPL_TC) return tc_workspace_bytes(p);
+    if (impl == PF_IMPL_TC_REFFLOW) return tc_refflow_workspace_bytes(p);
+    return simt_workspace_bytes(p);
 }
 
 bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
@@ -107,7 +115,7 @@ int forward(const pf_params* a) {
     p.O = a->O; p.S_final = a->S_final;
     p.stream = (cudaStream_t)a->stream;
 
-    const size_t need = impl == PF_IMPL_TC ? tc_workspace_bytes(p) : simt_workspace_bytes(p);
+    const size_t need = workspace_need(p, impl);
     void* ws = a->workspace;
     bool own = false;
     if (ws) {
@@ -118,7 +126,7 @@ int forward(const pf_params* a) {
     }
     g_launch_accum = 0;
     g_prof_n = 0;
-    st = impl == PF_IMPL_TC ? tc_forward(p, ws) : simt_forward(p, ws);
+    st = impl == PF_IMPL_TC ? tc_forward(p, ws) : impl == PF_IMPL_TC_REFFLOW ? tc_forward_refflow(p, ws) : simt_forward(p, ws);
     if (own) {
         cudaError_t e = cudaFreeAsync(ws, p.stream);
         if (e != cudaSuccess && st == PF_OK) st = record_cuda_error(e, "cudaFreeAsync");
@@ -165,7 +173,7 @@ size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chun
     pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
     const int sel = pf::select_impl(p, impl);
     if (sel < 0) return 0;
-    return sel == PF_IMPL_TC ? pf::tc_workspace_bytes(p) : pf::simt_workspace_bytes(p);
+    return pf::workspace_need(p, sel);
 }
 
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {

@@ -52,6 +52,7 @@ int simt_forward(const Problem& p, void* workspace);
 
 // tcgen05 path (pf_tc.cu)
 bool tc_supported(const Problem& p);
+bool tc_scan_supported(const Problem& p);
 size_t tc_workspace_bytes(const Problem& p);
 int tc_forward(const Problem& p, void* workspace);
 

@@ -11,6 +11,7 @@
 // Rows of a chunk are m = t*r + j (token t, factor j), n = chunk*r.  Rows past the end of the
 // sequence behave as beta = 0, k = 0, which leaves the state untouched; their outputs are not stored.
 #include "pf_common.cuh"
+#include "pf_tc.cuh"
 
 namespace pf {
 namespace {
@@ -363,7 +364,7 @@ Ws carve(const Problem& p, void* workspace) {
 }
 
 template <class Tin>
-int run(const Problem& p, void* workspace) {
+int run(const Problem& p, void* workspace, bool prepare_only) {
     Geo g{p.L, p.d_k, p.d_v, p.r, p.chunk, p.n(), p.chunks_per_seq()};
     const long long G = p.total_chunks();
     const long long nseq = (long long)p.B * p.H;
@@ -390,6 +391,11 @@ int run(const Problem& p, void* workspace) {
         prof_end(p.stream);
         launches += 3;
     }
+    if (prepare_only) {
+        PF_CUDA_TRY(cudaGetLastError());
+        count_launch(launches);
+        return PF_OK;
+    }
     // With L = 0 the scan still runs: it copies S0 to S_final.
     prof_begin("simt_scan", p.stream);
     simt_scan<Tin><<<(unsigned)(nseq * (p.d_v / DVS)), 256, scan_smem, p.stream>>>(q, k, p.S0, p.O, p.S_final, g, ws);
@@ -410,8 +416,17 @@ size_t simt_workspace_bytes(const Problem& p) {
 }
 
 int simt_forward(const Problem& p, void* workspace) {
-    if (p.in_dtype == PF_DTYPE_F32) return run<float>(p, workspace);
-    return run<__nv_bfloat16>(p, workspace);
+    if (p.in_dtype == PF_DTYPE_F32) return run<float>(p, workspace, false);
+    return run<__nv_bfloat16>(p, workspace, false);
+}
+
+int simt_prepare(const Problem& p, void* workspace, float** W, float** U, float** P) {
+    Ws ws = carve(p, workspace);
+    *W = ws.W;
+    *U = ws.U;
+    *P = ws.P;
+    if (p.in_dtype == PF_DTYPE_F32) return run<float>(p, workspace, true);
+    return run<__nv_bfloat16>(p, workspace, true);
 }
 
 }  // namespace pf

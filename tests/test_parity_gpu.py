@@ -164,3 +164,40 @@ def test_argument_errors_launch_nothing():
     assert rc == -1
     torch.cuda.synchronize()
     assert float(O.abs().sum()) == 0.0
+
+
+# --- tensor-core path -------------------------------------------------------------------------------
+
+TC_CASES = [
+    Workload("tc_r2_d128", B=1, H=2, L=512, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=31),
+    Workload("tc_r2_ragged", B=2, H=1, L=333, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=32),
+    Workload("tc_r1_d128", B=1, H=2, L=300, d_k=128, d_v=128, r=1, chunk=64, s0_std=0.1, seed=33),
+    Workload("tc_r4_d64_c32", B=2, H=2, L=200, d_k=64, d_v=64, r=4, chunk=32, beta_scale=2.0, seed=34),
+    Workload("tc_dk64_dv128", B=1, H=2, L=256, d_k=64, d_v=128, r=2, chunk=64, s0_std=0.1, seed=35),
+    Workload("tc_dk128_dv64", B=1, H=2, L=256, d_k=128, d_v=64, r=2, chunk=32, s0_std=0.1, seed=36),
+    Workload("tc_one_token", B=1, H=1, L=1, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=37),
+]
+
+
+def _run_with_status(w, impl):
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    need = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, impl)
+    assert need > 0
+    ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[off:off + need])
+    torch.cuda.synchronize()
+    status = int(ws[off:off + 4].view(torch.int32).item())
+    assert status == 0, f"device-side wait {status} expired"
+    O_ref, Sf_ref = util.run_oracle(inp)
+    return util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
+
+
+@pytest.mark.parametrize("w", TC_CASES, ids=lambda w: w.name)
+def test_tc_scan_with_reference_flows(w):
+    """tc_scan alone: the per-chunk flows come from the fp32 SIMT kernels."""
+    eo, es = _run_with_status(w, "tc_refflow")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
