@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
         mbar_init(&bar, 1);
         mbar_fence_init();
     }
+    __syncwarp();
     if (warp == 0) tmem_alloc(&tmem_base, 256);
     fence_async_smem();
     tc_fence_before();

@@ -201,3 +201,10 @@ def test_tc_scan_with_reference_flows(w):
     """tc_scan alone: the per-chunk flows come from the fp32 SIMT kernels."""
     eo, es = _run_with_status(w, "tc_refflow")
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+@pytest.mark.parametrize("w", TC_CASES, ids=lambda w: w.name)
+def test_tc_full_path(w):
+    """tc_flow + tc_scan: everything on tensor cores."""
+    eo, es = _run_with_status(w, "tc")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
