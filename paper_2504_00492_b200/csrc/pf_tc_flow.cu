@@ -136,6 +136,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
     __shared__ uint32_t tmem_base_s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = g.r, C = g.C;
+    const int dvs_shift = (dvs == 64) ? 6 : 5;
     int* err = ws.err;
 
     uint8_t* sKQ = smem + SM::kq_off;
@@ -176,6 +177,15 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     uint32_t tma_phase = 0, mma_phase = 0;
     bool ok = true;
+    // per-phase cycle counters of CTA 0 (diagnostic; words 32.. of the status block)
+    long long t_prev = clock64();
+    auto lap = [&](int phase) {
+        if (blockIdx.x == 0 && tid == 0) {
+            const long long now = clock64();
+            atomicAdd((unsigned long long*)(ws.err + 32) + phase, (unsigned long long)(now - t_prev));
+            t_prev = now;
+        }
+    };
 
     for (long long gc = blockIdx.x; gc < G && ok; gc += gridDim.x) {
         const long long seq = gc / g.NC;
@@ -203,6 +213,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         tma_phase ^= 1;
         if (!ok) break;
 
+        lap(0);
         // ---- bf16 -> fp16 in place (elementwise, so the swizzled layout is untouched) --------------------
         {
             constexpr int chunks = (SM::kq_bytes + SM::v_bytes) / 16;   // the two regions are contiguous
@@ -221,6 +232,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         fence_async_smem();
         __syncthreads();
 
+        lap(1);
         // ---- MMA1: [G | P0^T] = K [K;Q]^T ---------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -232,9 +244,11 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         if (!ok) break;
         tc_fence_after();
 
+        lap(2);
         // ---- epilogue 1: A -> X buffer (fp16) + fp32 diagonal blocks; P^T -> fp16 -------------------------
         {
             const int tokm = m / r;
+            const int row_lim = tokm * r;   // rows m' < row_lim belong to earlier tokens: tok(m') < tok(m)
 #pragma unroll
             for (int c0 = 0; c0 < N; c0 += 32) {
                 uint32_t rr[32];
@@ -247,7 +261,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const int mp = c0 + j8 + j;
-                            a[j] = (mp / r < tokm) ? beta_m * __uint_as_float(rr[j8 + j]) : 0.f;
+                            a[j] = (mp < row_lim) ? beta_m * __uint_as_float(rr[j8 + j]) : 0.f;
                         }
                         uint4 pk = make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                         *(uint4*)(sX + slab_off(m, c0 + j8, N)) = pk;
@@ -282,6 +296,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         tc_fence_before();
         __syncthreads();
 
+        lap(3);
         // ---- solve: 16x16 diagonal blocks by forward substitution (thread = one column of one block) ------
         if (tid < N) {
             const int b = tid >> 4, cc = tid & 15;
@@ -302,10 +317,12 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
                 *(__half*)(sX + slab_off(16 * b + mm, 16 * b + cc, N)) = __float2half_rn(x[mm]);
         }
         __syncthreads();
+        lap(4);
         merge_level<N, 16>(x_b, sX, warp, lane);
         merge_level<N, 32>(x_b, sX, warp, lane);
         if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
 
+        lap(5);
         // ---- T' = X diag(beta): the row owner scales its row by the column betas -----------------------------
         if (m < N) {
 #pragma unroll
@@ -323,6 +340,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         fence_async_smem();
         __syncthreads();
 
+        lap(6);
         // ---- MMA2: W = T' K,  Uh = T' V -------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -335,6 +353,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         if (!ok) break;
         tc_fence_after();
 
+        lap(7);
         // ---- epilogue 2: W and Uh as fp16 operands (Uh overwrites V) ----------------------------------
 #pragma unroll 1
         for (int c0 = 0; c0 < DK + DV; c0 += 32) {
@@ -358,6 +377,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         tc_fence_before();
         __syncthreads();
 
+        lap(8);
         // ---- MMA3: E = -K^T W, Xi = K^T Uh;  MMA4: Qt^T = Q^T - W^T P^T, O_intra^T = Uh^T P^T ---------------
         if (tid == 0) {
             tc_fence_after();
@@ -373,6 +393,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         if (!ok) break;
         tc_fence_after();
 
+        lap(9);
         // ---- epilogue 3: the chunk's flow -> workspace; O_intra -> O -----------------------------------
         {
             const int i = tid;   // accumulator lane: a d_k index (E, Xi, Qt^T) or a d_v index (O_intra^T)
@@ -395,7 +416,8 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
                             *(uint4*)(Eo + slab_off(i, c0 + j8, DK)) = pk;
                         } else {
                             const int j = c0 - DK + j8;
-                            *(uint4*)(Xo + ((size_t)(j / dvs) * DK * dvs + (size_t)i * dvs + (j % dvs)) * 2) = pk;
+                            const int sl = j >> dvs_shift, jj = j & (dvs - 1);
+                            *(uint4*)(Xo + ((size_t)sl * DK * dvs + (size_t)i * dvs + jj) * 2) = pk;
                         }
                     }
                 }
@@ -431,6 +453,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         tc_fence_before();
         __syncthreads();   // shared and tensor memory are reused by the next chunk
+        lap(10);
     }
     tc_fence_before();
     __syncthreads();
