@@ -85,6 +85,33 @@ int pf_deltanet_fwd_f32(const float* q, const float* k, const float* v, const fl
                         const float* S0, int B, int H, int L, int d_k, int d_v, int r, int chunk,
                         float* O, float* S_final, void* stream);
 
+/*
+ * pf_deltanet_fwd_f32_static -- pf_deltanet_fwd_f32 for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the fp32 path, same arithmetic.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaMallocAsync is off limits -- inside a region that
+ * must not touch the allocator (a real-time loop, a host that gave this library a fixed memory budget,
+ * a process whose device allocator belongs to another runtime).  The other entry points take their
+ * per-chunk scratch from the stream-ordered allocator or from the caller; this one uses a fixed array
+ * of PF_STATIC_SCRATCH_BYTES that is part of the library image, so it calls no allocating routine.
+ *
+ *   - Arguments, layouts, results and error codes are those of pf_deltanet_fwd_f32.
+ *   - A problem whose scratch (pf_workspace_bytes(..., PF_DTYPE_F32, PF_IMPL_SIMT)) exceeds
+ *     PF_STATIC_SCRATCH_BYTES is refused with PF_ERR_WORKSPACE and nothing is launched.
+ *   - The array occupies PF_STATIC_SCRATCH_BYTES on every GPU that loads the library, until exit.
+ *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
+ *     with that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the array and it keeps the previous call's contents.  Nothing in it
+ *     needs clearing (each call writes what it later reads), but two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it: serialise them.
+ */
+#define PF_STATIC_SCRATCH_BYTES (8u << 20)
+int pf_deltanet_fwd_f32_static(const float* q, const float* k, const float* v, const float* beta,
+                               const float* S0, int B, int H, int L, int d_k, int d_v, int r, int chunk,
+                               float* O, float* S_final, void* stream);
+/* The compiled-in value of PF_STATIC_SCRATCH_BYTES. */
+size_t pf_static_scratch_bytes(void);
+
 typedef struct pf_params {
     const void* q;            /* as in pf_deltanet_fwd, element type given by in_dtype */
     const void* k;

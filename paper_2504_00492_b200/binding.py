@@ -25,6 +25,7 @@ EXPORTS = [
     "pf_deltanet_fwd", "pf_deltanet_fwd_f32", "pf_deltanet_fwd_ex", "pf_workspace_bytes", "pf_select_impl",
     "pf_last_launch_count", "pf_status_string", "pf_last_error_string", "pf_version",
     "pf_profile_enable", "pf_profile_count", "pf_profile_read", "pf_tc_selftest",
+    "pf_deltanet_fwd_f32_static", "pf_static_scratch_bytes",
 ]
 
 
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.pf_profile_count.argtypes = []
         L.pf_profile_read.restype = ci
         L.pf_profile_read.argtypes = [ci, ctypes.c_char_p, ci, ctypes.POINTER(ctypes.c_float)]
+        L.pf_deltanet_fwd_f32_static.restype = ci
+        L.pf_deltanet_fwd_f32_static.argtypes = [vp] * 5 + [ci] * 7 + [vp, vp, vp]
+        L.pf_static_scratch_bytes.restype = ctypes.c_size_t
+        L.pf_static_scratch_bytes.argtypes = []
         L.pf_tc_selftest.restype = ci
         L.pf_tc_selftest.argtypes = [ci, vp, vp, vp, ci, vp]
         _lib = L
@@ -150,6 +155,26 @@ def pf_deltanet_fwd_f32(q, k, v, beta, S0, chunk: int, O=None, S_final=None, str
     if st != 0:
         raise PfError(st, "pf_deltanet_fwd_f32")
     return O, S_final
+
+
+def pf_deltanet_fwd_f32_static(q, k, v, beta, S0, chunk: int, O=None, S_final=None, stream=None,
+                               want_state: bool = True):
+    """pf_deltanet_fwd_f32 without any device allocation inside the library: the per-chunk scratch is a
+    fixed array of pf_static_scratch_bytes() built into libpf.so.  Pass O (and S_final) if the caller
+    must not allocate either; otherwise they are created here with torch.  Problems too large for the
+    fixed array raise PfError with status -6.  Calls on one device must not overlap on the GPU."""
+    B, H, L, d_k, d_v, r = _check_inputs(q, k, v, beta, S0, torch.float32)
+    O, S_final = _outputs(q, B, H, L, d_k, d_v, O, S_final, want_state)
+    with torch.cuda.device(q.device):
+        st = lib().pf_deltanet_fwd_f32_static(_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(S0), B, H, L, d_k, d_v, r,
+                                              chunk, _ptr(O), _ptr(S_final), _stream(stream))
+    if st != 0:
+        raise PfError(st, "pf_deltanet_fwd_f32_static")
+    return O, S_final
+
+
+def pf_static_scratch_bytes() -> int:
+    return int(lib().pf_static_scratch_bytes())
 
 
 def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Optional[torch.Tensor] = None,
