@@ -191,9 +191,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(pf_synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures)")
+    ap.add_argument("--heads", type=int, default=0, help="override H of the workload (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pf_synth.CONFIGS[args.workload]
+    if args.batch or args.heads:
+        w = w.with_(B=args.batch or w.B, H=args.heads or w.H)
+        w = w.with_(name=f"{w.name}[B={w.B},H={w.H}]")
 
     if args.impl == "reference":
         run_reference(args, w)
