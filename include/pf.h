@@ -59,10 +59,15 @@ enum { PF_DTYPE_BF16 = 0, PF_DTYPE_F32 = 1 };
 /* Which kernels evaluate the chunk form.
  *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
- *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.   */
+ *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.  For
+ *                  d_k = d_v = 128 with at most (SM count - 8) sequences this is ONE cooperative launch in
+ *                  which flow-building CTAs and state-scanning CTAs run side by side; other shapes take
+ *                  the two-launch form below.   */
 enum { PF_IMPL_AUTO = 0, PF_IMPL_SIMT = 1, PF_IMPL_TC = 2,
        /* diagnostic: per-chunk flows built by the fp32 SIMT kernels, state scan on tensor cores */
-       PF_IMPL_TC_REFFLOW = 3 };
+       PF_IMPL_TC_REFFLOW = 3,
+       /* tensor-core path as two launches (all flows, then the scan), whatever the shape */
+       PF_IMPL_TC_SPLIT = 4 };
 
 /*
  * pf_deltanet_fwd -- the central call: bf16 inputs, fp32 accumulation, fp32 outputs.

@@ -18,7 +18,9 @@ LIB_PATH = os.path.join(_PKG, "libpf.so")
 PF_DTYPE_BF16, PF_DTYPE_F32 = 0, 1
 PF_IMPL_AUTO, PF_IMPL_SIMT, PF_IMPL_TC = 0, 1, 2
 PF_IMPL_TC_REFFLOW = 3
-IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC, "tc_refflow": PF_IMPL_TC_REFFLOW}
+PF_IMPL_TC_SPLIT = 4
+IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC, "tc_refflow": PF_IMPL_TC_REFFLOW,
+                "tc_split": PF_IMPL_TC_SPLIT}
 
 # every symbol include/pf.h declares
 EXPORTS = [

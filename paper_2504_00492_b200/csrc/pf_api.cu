@@ -70,13 +70,15 @@ int select_impl(const Problem& p, int impl) {
         case PF_IMPL_SIMT: return PF_IMPL_SIMT;
         case PF_IMPL_TC: return tc_supported(p) ? (int)PF_IMPL_TC : (int)PF_ERR_UNSUPPORTED;
         case PF_IMPL_AUTO: return tc_supported(p) ? PF_IMPL_TC : PF_IMPL_SIMT;
+        case PF_IMPL_TC_SPLIT: return tc_supported(p) ? (int)PF_IMPL_TC_SPLIT : (int)PF_ERR_UNSUPPORTED;
         case PF_IMPL_TC_REFFLOW: return tc_scan_supported(p) ? (int)PF_IMPL_TC_REFFLOW : (int)PF_ERR_UNSUPPORTED;
         default: return PF_ERR_UNSUPPORTED;
     }
 }
 
 size_t workspace_need(const Problem& p, int impl) {
-    if (impl == PF_IMPL_TC) return tc_workspace_bytes(p);
+    if (impl == PF_IMPL_TC) return fused_supported(p) ? fused_workspace_bytes(p) : tc_workspace_bytes(p);
+    if (impl == PF_IMPL_TC_SPLIT) return tc_workspace_bytes(p);
     if (impl == PF_IMPL_TC_REFFLOW) return tc_refflow_workspace_bytes(p);
     return simt_workspace_bytes(p);
 }
@@ -126,7 +128,10 @@ int forward(const pf_params* a) {
     }
     g_launch_accum = 0;
     g_prof_n = 0;
-    st = impl == PF_IMPL_TC ? tc_forward(p, ws) : impl == PF_IMPL_TC_REFFLOW ? tc_forward_refflow(p, ws) : simt_forward(p, ws);
+    if (impl == PF_IMPL_TC) st = fused_supported(p) ? fused_forward(p, ws) : tc_forward(p, ws);
+    else if (impl == PF_IMPL_TC_SPLIT) st = tc_forward(p, ws);
+    else if (impl == PF_IMPL_TC_REFFLOW) st = tc_forward_refflow(p, ws);
+    else st = simt_forward(p, ws);
     if (own) {
         cudaError_t e = cudaFreeAsync(ws, p.stream);
         if (e != cudaSuccess && st == PF_OK) st = record_cuda_error(e, "cudaFreeAsync");

@@ -29,6 +29,11 @@ int tc_scan_launch(const Problem& p, const TcWs& ws);
 int tc_forward_refflow(const Problem& p, void* workspace);
 size_t tc_refflow_workspace_bytes(const Problem& p);
 
+// pf_fused.cu: flow builders and state scan in one cooperative launch
+bool fused_supported(const Problem& p);
+size_t fused_workspace_bytes(const Problem& p);
+int fused_forward(const Problem& p, void* workspace);
+
 // pf_simt.cu: runs the gram/solve/wu kernels only and returns where W, Uh and P were left.
 int simt_prepare(const Problem& p, void* workspace, float** W, float** U, float** P);
 
