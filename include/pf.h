@@ -146,6 +146,12 @@ size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chun
 /* Which PF_IMPL_* pf_deltanet_fwd_ex would run for this problem (negative pf_status if none). */
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
 
+/* Tuning knobs (process-wide, not thread-safe; results do not depend on them).  Returns PF_OK,
+ * PF_ERR_UNSUPPORTED for an unknown name, PF_ERR_INVALID for a value out of range.
+ *   "ring_depth" (3..64, default 8): slots per sequence of the L2-resident ring through which the
+ *       single-launch tensor-core path hands each chunk's flow to the state scan. */
+int pf_set_option(const char* name, int value);
+
 /* Number of kernels the last successful call on this host thread enqueued. */
 int pf_last_launch_count(void);
 

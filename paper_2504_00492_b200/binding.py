@@ -27,7 +27,7 @@ EXPORTS = [
     "pf_deltanet_fwd", "pf_deltanet_fwd_f32", "pf_deltanet_fwd_ex", "pf_workspace_bytes", "pf_select_impl",
     "pf_last_launch_count", "pf_status_string", "pf_last_error_string", "pf_version",
     "pf_profile_enable", "pf_profile_count", "pf_profile_read", "pf_tc_selftest",
-    "pf_deltanet_fwd_f32_static", "pf_static_scratch_bytes",
+    "pf_deltanet_fwd_f32_static", "pf_static_scratch_bytes", "pf_set_option",
 ]
 
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.pf_deltanet_fwd_f32_static.argtypes = [vp] * 5 + [ci] * 7 + [vp, vp, vp]
         L.pf_static_scratch_bytes.restype = ctypes.c_size_t
         L.pf_static_scratch_bytes.argtypes = []
+        L.pf_set_option.restype = ci
+        L.pf_set_option.argtypes = [ctypes.c_char_p, ci]
         L.pf_tc_selftest.restype = ci
         L.pf_tc_selftest.argtypes = [ci, vp, vp, vp, ci, vp]
         _lib = L
@@ -212,6 +214,12 @@ def pf_workspace_bytes(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl
 def pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
     impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
     return int(lib().pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype, impl))
+
+
+def pf_set_option(name: str, value: int) -> None:
+    st = lib().pf_set_option(name.encode(), int(value))
+    if st != 0:
+        raise PfError(st, f"pf_set_option({name!r})")
 
 
 def pf_last_launch_count() -> int:

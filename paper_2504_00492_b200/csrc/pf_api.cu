@@ -189,6 +189,11 @@ int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
 
 int pf_last_launch_count(void) { return pf::g_launches; }
 
+int pf_set_option(const char* name, int value) {
+    if (!name) return PF_ERR_INVALID;
+    return pf::fused_set_option(name, value);
+}
+
 void pf_profile_enable(int on) { pf::g_prof_on = on != 0; }
 
 int pf_profile_count(void) { return pf::g_prof_n; }

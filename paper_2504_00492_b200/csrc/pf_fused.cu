@@ -17,19 +17,26 @@
 // The ring (R slots of 112 KB per sequence) is rewritten in place, so the hand-off never has to reach HBM:
 // the only compulsory HBM traffic is one read of q, k, v, beta and one write of O.
 //
-// A flow CTA is software-pipelined over two chunks with five kinds of warps (14 warps):
+// A flow CTA is software-pipelined over two chunks (15 warps):
 //   warps 0-3  "solve"  epilogue of G = K K^T (mask, column scaling, fp16) and the triangular inverse
-//   warps 4-7  "mid"    bf16 -> fp16 conversion of K, V, Q; epilogue of P^T; epilogue of [W | Uh]
-//   warps 8-11 "out"    epilogue of [E | Xi] and [Qt^T | OI^T], staging and bulk stores into the ring
+//   warps 4-7  "mid"    epilogues of [Uh | W] and P^T; bf16 -> fp16 conversion of K, V, Q
+//   warps 8-11 "out"    epilogues of [E | Xi] (staged, bulk-stored) and [Qt^T | OI^T] (stored directly)
 //   warp 12             TMA loads (K and V double-buffered, Q single)
-//   warp 13             tcgen05.mma issue
-// Tensor memory: RA = columns [0,256) holds [W | Uh] and then [E | Xi]; RB = [256,384) holds G of the NEXT
+//   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
+//   warp 14             bulk stores into the ring, ring back-pressure, ready flags
+// Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi]; RB = [256,384) holds G of the NEXT
 // chunk and then [Qt^T | OI^T] of the current one; RC = [384,448) holds P0^T.
+// G is formed from the bf16 tiles as they land (both operands raw); every other product has a derived fp16
+// operand, so K, V and Q are converted to fp16 in place, off the critical path.
 //
-// A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns),
-// warps 8-11 add OI and write O, warp 12 streams E/Qt images in with bulk copies, warp 13 issues the MMAs.
+// A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns; the
+// first warp of each half issues that half's Delta MMAs), warps 8-11 add OI and write O, warp 12 streams
+// the E / Xi / Qt images in with bulk copies, warp 13 issues the O^T MMAs and reports consumed chunks.
 //
-// Every wait is bounded (about a second of cycles) and reports a code in the status word.
+// Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
+// deliberately kept rolled: the instruction footprint of fifteen differently-specialised warps matters.
+#include <string.h>
+
 #include "pf_common.cuh"
 #include "pf_tc.cuh"
 #include "pf_tc_prims.cuh"
@@ -40,9 +47,8 @@ using namespace tc;
 
 namespace {
 
-constexpr int FT = 448;                 // threads per CTA
+constexpr int FT = 480;                 // threads per CTA
 constexpr int DK = 128, DV = 128;
-constexpr int SCAN_STAGES = 3;
 
 // ---- ring slot layout (bytes) ---------------------------------------------------------------------------
 constexpr uint32_t SLOT_E = 0;                          // E image : fp16 [2 slabs][128 rows i][128 B]   (K-major A)
@@ -69,53 +75,94 @@ struct FusedMaps {
 };
 
 // ---- shared memory ----------------------------------------------------------------------------------------
-// flow role
-constexpr int F_K = 0;                          // 2 x 32 KB  K (fp16 after conversion)
-constexpr int F_V = F_K + 2 * 32768;            // 2 x 32 KB  V -> Uh -> Xi staging
-constexpr int F_X = F_V + 2 * 32768;            // 2 x 32 KB  A -> X -> W -> E staging
-constexpr int F_Q = F_X + 2 * 32768;            // 16 KB      Q
-constexpr int F_PT = F_Q + 16384;               // 16 KB      P^T -> Qt staging
+// flow role: two 96 KB regions (chunk parity), each holding  X/W | V/Uh | K  back to back (n*256 bytes each),
+// so that [V | K] and [W | Uh] are single 256-column B operands.  After the chunk's last MMA the region is
+// staging space: the E image at +0, the Xi image at +32 KB.
+constexpr int F_REGION = 98304;
+constexpr int F_STAGE_XI = 32768;
+constexpr int F_Q = 2 * F_REGION;               // 16 KB      Q
+constexpr int F_PT = F_Q + 16384;               // 16 KB      P^T
 constexpr int F_BETA = F_PT + 16384;            // 2 x 128 fp32
 constexpr int F_BAR = F_BETA + 1024;
 constexpr int SMEM_BYTES = F_BAR + 512;         // 230912
 // scan role
-constexpr int S_STAGE = 0;                      // 3 x (32 KB E + 16 KB Qt)
-constexpr int S_STAGE_BYTES = 32768 + 16384;
-constexpr int S_S16 = S_STAGE + SCAN_STAGES * S_STAGE_BYTES;   // 2 x 32 KB fp16 copy of the state
+constexpr int S_E = 0;                          // 2 x 32 KB  E images
+constexpr int S_XI = S_E + 2 * 32768;           // 2 x 32 KB  Xi images
+constexpr int S_QT = S_XI + 2 * 32768;          // 2 x 16 KB  Qt images
+constexpr int S_S16 = S_QT + 2 * 16384;         // 2 x 32 KB  fp16 copies of the state
 static_assert(S_S16 + 2 * 32768 <= F_BAR, "scan role fits below the barrier block");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // barriers (indices into the uint64_t block at F_BAR)
 enum {
     // flow role
-    B_KFULL = 0,      // [2] TMA: K landed
+    B_KFULL = 0,      // [2] TMA: K landed (bf16)
     B_VFULL = 2,      // [2]
     B_QFULL = 4,
-    B_K16 = 5,        // [2] mid: K converted
+    B_K16 = 5,        // [2] mid: K converted to fp16
     B_V16 = 7,        // [2]
     B_Q16 = 9,
     B_GDONE = 10,     // mma: G complete
     B_GFREE = 11,     // solve: G drained from tensor memory
     B_XREADY = 12,    // [2] solve: X complete
-    B_D2DONE = 14,    // mma: [W | Uh] complete
+    B_D2DONE = 14,    // mma: [Uh | W] complete
     B_WUREADY = 15,   // mid: W, Uh in shared memory (RA drained)
     B_P0DONE = 16,    // mma: P0^T complete
     B_PTREADY = 17,   // mid: P^T in shared memory (RC drained)
     B_D34DONE = 18,   // mma: [E | Xi] and [Qt^T | OI^T] complete
-    B_D4FREE = 19,    // out: RB drained, Q no longer needed
+    B_D4FREE = 19,    // out: RB drained
     B_RAFREE = 20,    // out: RA drained
-    B_XFREE = 21,     // [2] out: bulk store finished reading the E staging
-    B_VFREE = 23,     // [2] out: ... the Xi staging
-    B_PTFREE = 25,    // out: ... the Qt staging
+    B_XFREE = 21,     // [2] store warp: bulk store finished reading the E staging
+    B_VFREE = 23,     // [2] store warp: ... the Xi staging
+    B_QCOPIED = 25,   // out: Q copied into registers
+    B_STAGED = 26,    // out: E and Xi images staged
+    B_OUTDONE = 27,   // out: Qt and OI stored
+    B_SLOTOK = 28,    // store warp: the chunk's ring slot may be written
     // scan role
-    B_FULL = 32,      // [3] producer: E, Qt landed (and the slot's Xi, OI are visible)
-    B_EMPTY = 35,     // [3] everyone is done with the stage's chunk
-    B_SREADY = 38,    // [2 buffers][2 halves]
-    B_DDONE = 42,     // [2 halves]
-    B_ODONE = 44,     // [2]
-    B_OFREE = 46,     // [2]
-    B_COUNT = 48
+    B_EFULL = 32,     // [2] producer: E image landed
+    B_EEMPTY = 34,    // [2] chain: both Delta halves of that chunk complete (two commits)
+    B_XIFULL = 36,    // [2] producer: Xi image landed
+    B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
+    B_QTFULL = 40,    // [2] producer: Qt image landed
+    B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
+    B_SREADY = 44,    // [2 buffers] chain: fp16 copy of the state published (256 arrivals)
+    B_S16FREE = 46,   // [2 buffers] mma: the O^T MMA that reads the copy is complete
+    B_DDONE = 48,     // [2 halves] Delta half complete
+    B_ODONE = 50,     // [2] mma: O^T complete
+    B_OFREE = 52,     // [2] output warps: O^T drained
+    B_COUNT = 54
 };
+
+// Diagnostic builds (-DPF_TIMING): chosen threads of flow CTA 0 and of scan CTA 0 accumulate the cycles they
+// spend in each wait (indexed by the wait's code) and in each lap, in the 64-bit words that follow the first
+// 1 KB of the status block.  Otherwise null, and the accounting compiles away.
+__device__ __forceinline__ unsigned long long* timing_slot(const FusedWs& ws, bool chosen) {
+#ifdef PF_TIMING
+    return chosen ? (unsigned long long*)(ws.status + 256) : nullptr;
+#else
+    (void)ws; (void)chosen;
+    return nullptr;
+#endif
+}
+#ifdef PF_TIMING
+#define PF_LAP(slot)                                                              \
+    do {                                                                          \
+        if (tim) {                                                                \
+            const long long n_ = clock64();                                       \
+            atomicAdd(tim + (slot), (unsigned long long)(n_ - t_lap));            \
+            t_lap = n_;                                                           \
+        }                                                                         \
+    } while (0)
+#else
+#define PF_LAP(slot) do { } while (0)
+#endif
+
+#define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code, tim)
+
+// byte offset of the 16-byte chunk `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
+__device__ __forceinline__ uint32_t chunk_off(int row, int col8, int R) {
+    return (uint32_t)(col8 >> 3) * (uint32_t)R * 128u + (uint32_t)row * 128u + ((((uint32_t)col8 & 7u) ^ ((uint32_t)row & 7u)) << 4);
+}
 
 __device__ __forceinline__ uint4 pack8(const uint32_t* r, float scale) {
     return make_uint4(pack_h2(__uint_as_float(r[0]) * scale, __uint_as_float(r[1]) * scale),
@@ -125,7 +172,7 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* r, float scale) {
 }
 
 // bf16 -> fp16 in place, elementwise (so the swizzled layout is untouched); 128 threads
-__device__ __forceinline__ void cvt_region(uint8_t* base, int bytes, int t128) {
+static __device__ __noinline__ void cvt_region(uint8_t* base, int bytes, int t128) {
     uint4* p = (uint4*)base;
     const int chunks = bytes >> 4;
 #pragma unroll 4
@@ -153,23 +200,25 @@ __device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, 
     const bool has_task = warp < TASKS;
     const int q = warp / STRIPS, strip = warp % STRIPS;
     const int lo0 = 2 * S * q, hi0 = lo0 + S, R0 = hi0 + 16 * strip;
+    const int id = lane >> 3;
     if (has_task) {
         float u[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) u[nt][e] = 0.f;
+        // (all column offsets below are multiples of 8, all row offsets multiples of 8 plus a lane term)
+        const int a_row = R0 + (lane & 15), a_c8 = (hi0 >> 3) + (lane >> 4);
+        const int b_rowl = (lane & 7) + ((id & 1) << 3), b_c8l = (id >> 1);
 #pragma unroll
         for (int kk = 0; kk < S / 16; ++kk) {
             if (kk > strip) continue;   // X_hi,hi is lower triangular
             uint32_t a[4];
-            ldmatrix_x4(a, xb + slab_off(R0 + (lane & 15), hi0 + 16 * kk + ((lane >> 4) << 3), N));
+            ldmatrix_x4(a, xb + chunk_off(a_row, a_c8 + 2 * kk, N));
 #pragma unroll
             for (int np = 0; np < S / 16; ++np) {
                 uint32_t b[4];
-                const int id = lane >> 3;
-                ldmatrix_x4_trans(b, xb + slab_off(hi0 + 16 * kk + (lane & 7) + ((id & 1) << 3),
-                                                   lo0 + 16 * np + ((id >> 1) << 3), N));
+                ldmatrix_x4_trans(b, xb + chunk_off(hi0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
                 mma_16816(u[2 * np], a, b[0], b[1]);
                 mma_16816(u[2 * np + 1], a, b[2], b[3]);
             }
@@ -189,9 +238,7 @@ __device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, 
             for (int np = 0; np < S / 16; ++np) {
                 if (np > kk) continue;  // X_lo,lo is lower triangular
                 uint32_t b[4];
-                const int id = lane >> 3;
-                ldmatrix_x4_trans(b, xb + slab_off(lo0 + 16 * kk + (lane & 7) + ((id & 1) << 3),
-                                                   lo0 + 16 * np + ((id >> 1) << 3), N));
+                ldmatrix_x4_trans(b, xb + chunk_off(lo0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
                 mma_16816(z[2 * np], a, b[0], b[1]);
                 mma_16816(z[2 * np + 1], a, b[2], b[3]);
             }
@@ -202,9 +249,9 @@ __device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, 
         const int gq = lane >> 2, t4 = lane & 3;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const int col = lo0 + 8 * nt + 2 * t4;
-            *(uint32_t*)(xg + slab_off(R0 + gq, col, N)) = pack_h2(-z[nt][0], -z[nt][1]);
-            *(uint32_t*)(xg + slab_off(R0 + gq + 8, col, N)) = pack_h2(-z[nt][2], -z[nt][3]);
+            const int c8 = (lo0 >> 3) + nt;
+            *(uint32_t*)(xg + chunk_off(R0 + gq, c8, N) + 4 * t4) = pack_h2(-z[nt][0], -z[nt][1]);
+            *(uint32_t*)(xg + chunk_off(R0 + gq + 8, c8, N) + 4 * t4) = pack_h2(-z[nt][2], -z[nt][3]);
         }
     }
     named_bar(1, 128);
@@ -220,11 +267,17 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = g.r, C = g.C, nseq = g.nseq;
     int* err = ws.status;
+    unsigned long long* const tim =
+        timing_slot(ws, fid == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416 || tid == 448));
+    const long long t_role = clock64();
+    long long t_lap = t_role;
+    (void)t_lap;
     const int nk = fid < g.items ? (g.items - fid + g.n_flow - 1) / g.n_flow : 0;
     const uint32_t RA = tb, RB = tb + 256, RC = tb + 384;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     constexpr uint32_t KV_SLAB = N * 128;                 // bytes of one 64-column slab of K / V / W / Uh
     constexpr uint32_t K_BYTES = N * 256;
+    constexpr int X_OFF = 0, V_OFF = N * 256, K_OFF = 2 * N * 256;   // inside a parity region
 
     auto item = [&](int k, int& seq, int& c) {
         const int q = fid + k * g.n_flow;
@@ -235,7 +288,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     if (warp < 4) {
         // ------------------------------------------------ solve: G epilogue + triangular inverse -------------
         const int m = tid;
-        const int tokm = m / r, row_lim = tokm * r;       // rows m' < row_lim belong to earlier tokens
+        const int row_lim = (m / r) * r;       // rows m' < row_lim belong to earlier tokens
         float* sBeta = (float*)(smem + F_BETA);
         float beta_next = 0.f;
         if (nk > 0) {
@@ -244,9 +297,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             const int nv = min(C, g.L - c * C) * r;
             if (m < nv) beta_next = __bfloat162float(beta[((long long)seq * g.L + (long long)c * C) * r + m]);
         }
+#pragma unroll 1
         for (int k = 0; k < nk; ++k) {
             const int b = k & 1;
-            uint8_t* sX = smem + F_X + b * 32768;
+            uint8_t* sX = smem + b * F_REGION + X_OFF;
             const uint32_t x_b = smem_u32(sX);
             float* sB = sBeta + b * 128;
             const float bm = beta_next;
@@ -260,47 +314,51 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
             bool ok = true;
-            if (k >= 2) ok = mbar_wait_clk(&bar[B_XFREE + b], ((k >> 1) - 1) & 1, err, 101);
+            if (k >= 2) ok = PF_WAIT(B_XFREE + b, ((k >> 1) - 1) & 1, 101);
             sB[m] = bm;     // the readers of this half (chunk k-2) are done: X of chunk k-2 has been released
-            ok = ok && mbar_wait_clk(&bar[B_GDONE], k & 1, err, 102);
+            ok = ok && PF_WAIT(B_GDONE, k & 1, 102);
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
-            // A = Mstrict (.) (G diag(beta)) as fp16 into X
-#pragma unroll
+            PF_LAP(1);
+            // A = Mstrict (.) (G diag(beta)) as fp16 into X; column groups right of the warp's rows are zero
+#pragma unroll 1
             for (int c0 = 0; c0 < N; c0 += 32) {
-                if (c0 < 32 * (warp + 1)) {
-                    uint32_t rr[32];
+                uint32_t rr[32];
+                const bool live = c0 < 32 * (warp + 1);
+                if (live) {
                     tmem_ld32(RB + lane_base + c0, rr);
                     tmem_ld_wait();
-                    if (m < N) {
+                }
+                if (m < N) {
 #pragma unroll
-                        for (int j8 = 0; j8 < 32; j8 += 8) {
+                    for (int j8 = 0; j8 < 32; j8 += 8) {
+                        uint4 pk = make_uint4(0, 0, 0, 0);
+                        if (live) {
+                            const float4 b0 = *(const float4*)(sB + c0 + j8), b1 = *(const float4*)(sB + c0 + j8 + 4);
+                            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                             float a[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int mp = c0 + j8 + j;
-                                a[j] = (mp < row_lim) ? sB[mp] * __uint_as_float(rr[j8 + j]) : 0.f;
-                            }
-                            *(uint4*)(sX + slab_off(m, c0 + j8, N)) =
-                                make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
+                            for (int j = 0; j < 8; ++j) a[j] = (c0 + j8 + j < row_lim) ? bb[j] * __uint_as_float(rr[j8 + j]) : 0.f;
+                            pk = make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                         }
+                        *(uint4*)(sX + chunk_off(m, (c0 + j8) >> 3, N)) = pk;
                     }
-                } else if (m < N) {
-#pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8) *(uint4*)(sX + slab_off(m, c0 + j8, N)) = make_uint4(0, 0, 0, 0);
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_GFREE]);
             named_bar(1, 128);
+            PF_LAP(2);
             // 16x16 diagonal blocks: forward substitution, one thread per column of one block (fp32)
             float x[16];
             const int bk = tid >> 4, cc = tid & 15;
             if (tid < N) {
+                const uint8_t* blk = sX + (bk >> 2) * (N * 128) + (16 * bk) * 128;    // row 16*bk of the block's slab
+                const int c8 = (2 * bk) & 7;                                          // first 16-byte chunk of the block
 #pragma unroll
                 for (int mm = 0; mm < 16; ++mm) {
-                    const uint4 lo = *(const uint4*)(sX + slab_off(16 * bk + mm, 16 * bk, N));
-                    const uint4 hi = *(const uint4*)(sX + slab_off(16 * bk + mm, 16 * bk + 8, N));
+                    const uint4 lo = *(const uint4*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4));
+                    const uint4 hi = *(const uint4*)(blk + mm * 128 + (((c8 + 1) ^ (mm & 7)) << 4));
                     const __half2* hl = (const __half2*)&lo;
                     const __half2* hh = (const __half2*)&hi;
                     float a[16];
@@ -320,59 +378,79 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             named_bar(1, 128);
             if (tid < N) {
+                uint8_t* blk = sX + (bk >> 2) * (N * 128) + (16 * bk) * 128;
+                const int c8 = ((2 * bk) & 7) + (cc >> 3);
 #pragma unroll
                 for (int mm = 0; mm < 16; ++mm)
-                    *(__half*)(sX + slab_off(16 * bk + mm, 16 * bk + cc, N)) = __float2half_rn(x[mm]);
+                    *(__half*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4) + (cc & 7) * 2) = __float2half_rn(x[mm]);
             }
             named_bar(1, 128);
+            PF_LAP(3);
             merge_level<N, 16>(x_b, sX, warp, lane);
             merge_level<N, 32>(x_b, sX, warp, lane);
             if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
             fence_async_smem();
             mbar_arrive(&bar[B_XREADY + b]);
+            PF_LAP(4);
         }
     } else if (warp < 8) {
-        // ------------------------------------------------ mid: conversions, P^T and [W | Uh] epilogues --------
+        // ------------------------------------------------ mid: [Uh | W] and P^T epilogues, conversions --------
         const int m = tid - 128;
         const int tokm = m / r;
         const float* sBeta = (const float*)(smem + F_BETA);
         uint8_t* sPT = smem + F_PT;
         if (nk > 0) {
-            if (!mbar_wait_clk(&bar[B_KFULL + 0], 0, err, 111)) return;
-            cvt_region(smem + F_K, K_BYTES, m);
+            // chunk 0: K after its Gram product has read the bf16 tile, V and Q as they land
+            if (!PF_WAIT(B_KFULL + 0, 0, 111) || !PF_WAIT(B_GDONE, 0, 110)) return;
+            cvt_region(smem + K_OFF, K_BYTES, m);
             fence_async_smem();
             mbar_arrive(&bar[B_K16 + 0]);
-            if (!mbar_wait_clk(&bar[B_VFULL + 0], 0, err, 112)) return;
-            cvt_region(smem + F_V, K_BYTES, m);
+            if (!PF_WAIT(B_VFULL + 0, 0, 112)) return;
+            cvt_region(smem + V_OFF, K_BYTES, m);
             fence_async_smem();
             mbar_arrive(&bar[B_V16 + 0]);
+            if (!PF_WAIT(B_QFULL, 0, 109)) return;
+            cvt_region(smem + F_Q, 16384, m);
+            fence_async_smem();
+            mbar_arrive(&bar[B_Q16]);
         }
+#pragma unroll 1
         for (int k = 0; k < nk; ++k) {
             const int b = k & 1, b1 = b ^ 1;
             int seq, c;
             item(k, seq, c);
             const int Cv = min(C, g.L - c * C), nv = Cv * r;
-            if (k + 1 < nk) {
-                if (!mbar_wait_clk(&bar[B_KFULL + b1], ((k + 1) >> 1) & 1, err, 113)) return;
-                cvt_region(smem + F_K + b1 * 32768, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_K16 + b1]);
-            }
-            if (!mbar_wait_clk(&bar[B_QFULL], k & 1, err, 114)) return;
-            cvt_region(smem + F_Q, 16384, m);
-            fence_async_smem();
-            mbar_arrive(&bar[B_Q16]);
-            if (k + 1 < nk) {
-                if (!mbar_wait_clk(&bar[B_VFULL + b1], ((k + 1) >> 1) & 1, err, 115)) return;
-                cvt_region(smem + F_V + b1 * 32768, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_V16 + b1]);
-            }
-            // P^T = P0^T (.) Mincl as fp16 [m rows][64 t]
-            if (k >= 1 && !mbar_wait_clk(&bar[B_PTFREE], (k - 1) & 1, err, 116)) return;
-            if (!mbar_wait_clk(&bar[B_P0DONE], k & 1, err, 117)) return;
+            // ---- RA = X [V | K]:  Uh = diag(beta) (X V) over V,  -W = -diag(beta) (X K) over X, fp16 operands
+            if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
             tc_fence_after();
+            PF_LAP(12);
+            {
+                const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
+                uint8_t* sU = smem + b * F_REGION + V_OFF;
+                uint8_t* sW = smem + b * F_REGION + X_OFF;
+#pragma unroll 1
+                for (int c0 = 0; c0 < DV + DK; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RA + lane_base + c0, rr);
+                    tmem_ld_wait();
+                    if (m < N) {
+                        uint8_t* dst = (c0 < DV) ? sU : sW;
+                        const int col8 = ((c0 < DV) ? c0 : c0 - DV) >> 3;
+                        const float sc = (c0 < DV) ? bm : -bm;
 #pragma unroll
+                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + chunk_off(m, col8 + j8, N)) = pack8(rr + 8 * j8, sc);
+                    }
+                }
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(&bar[B_WUREADY]);
+            PF_LAP(13);
+            // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
+            if (k >= 1 && !PF_WAIT(B_D34DONE, (k - 1) & 1, 116)) return;
+            if (!PF_WAIT(B_P0DONE, k & 1, 117)) return;
+            tc_fence_after();
+#pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(RC + lane_base + c0, rr);
@@ -386,7 +464,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                             const int t = c0 + j8 + j;
                             a[j] = (tokm <= t && t < Cv && m < nv) ? __uint_as_float(rr[j8 + j]) : 0.f;
                         }
-                        *(uint4*)(sPT + m * 128 + ((((c0 + j8) >> 3) ^ (m & 7)) << 4)) =
+                        *(uint4*)(sPT + chunk_off(m, (c0 + j8) >> 3, N)) =
                             make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                     }
                 }
@@ -394,191 +472,234 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_PTREADY]);
-            // W = diag(beta) (X K), Uh = diag(beta) (X V) as fp16 operands (W over X, Uh over V)
-            if (!mbar_wait_clk(&bar[B_D2DONE], k & 1, err, 118)) return;
-            tc_fence_after();
-            const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
-            uint8_t* sW = smem + F_X + b * 32768;
-            uint8_t* sU = smem + F_V + b * 32768;
-#pragma unroll 2
-            for (int c0 = 0; c0 < DK + DV; c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(RA + lane_base + c0, rr);
-                tmem_ld_wait();
-                if (m < N) {
-                    uint8_t* dst = (c0 < DK) ? sW : sU;
-                    const int col0 = (c0 < DK) ? c0 : c0 - DK;
-#pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8) *(uint4*)(dst + slab_off(m, col0 + j8, N)) = pack8(rr + j8, bm);
-                }
+            PF_LAP(11);
+            // ---- conversions for chunk k+1 (K only once its Gram product has read the bf16 tile)
+            if (k + 1 < nk) {
+                if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
+                PF_LAP(14);
+                cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
+                fence_async_smem();
+                mbar_arrive(&bar[B_K16 + b1]);
+                PF_LAP(15);
+                if (!PF_WAIT(B_QFULL, (k + 1) & 1, 114)) return;
+                PF_LAP(16);
+                cvt_region(smem + F_Q, 16384, m);
+                fence_async_smem();
+                mbar_arrive(&bar[B_Q16]);
+                PF_LAP(17);
+                if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
+                PF_LAP(18);
+                cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
+                fence_async_smem();
+                mbar_arrive(&bar[B_V16 + b1]);
+                PF_LAP(19);
             }
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive(&bar[B_WUREADY]);
         }
     } else if (warp < 12) {
         // ------------------------------------------------ out: flow -> ring -----------------------------------
         const int i = tid - 256;
-        uint8_t* sQ = smem + F_Q;
-        uint8_t* sPT = smem + F_PT;
+        const uint8_t* sQ = smem + F_Q;
+#pragma unroll 1
         for (int k = 0; k < nk; ++k) {
             const int b = k & 1;
             int seq, c;
             item(k, seq, c);
             const int Cv = min(C, g.L - c * C);
-            const int slot_i = c % g.R;
-            uint8_t* slot = ws.ring + ((size_t)seq * g.R + slot_i) * SLOT_BYTES;
-            // the scan must be done with the chunk that used this slot before
-            bool ok = true;
-            if (c >= g.R && i == 0) ok = flag_wait_ge(&ws.consumed[seq], c - g.R + 1, err, 121);
-            ok = ok && mbar_wait_clk(&bar[B_Q16], k & 1, err, 122);
-            ok = ok && mbar_wait_clk(&bar[B_D34DONE], k & 1, err, 123);
-            tc_fence_after();
-            if (!named_bar_and(3, 128, ok)) return;
-            uint8_t* sE = smem + F_X + b * 32768;
-            uint8_t* sXi = smem + F_V + b * 32768;
-            // [Qt^T | OI^T] from RB:  Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t]  -> staging (over P^T);  OI -> ring
+            uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
+            // ---- column i of Q (fp16) into registers, so that the Q buffer can take the next chunk early
+            if (!PF_WAIT(B_Q16, k & 1, 122)) return;
+            uint32_t qreg[32];
+            {
+                const uint8_t* qcol = sQ + (i >> 6) * 8192 + (i & 7) * 2;
+                const int ci = (i & 63) >> 3;
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(RB + lane_base + c0, rr);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j8 = 0; j8 < 32; j8 += 8) {
-                    float a[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int t = c0 + j8 + j;
-                        a[j] = __uint_as_float(rr[j8 + j]) + __half2float(*(const __half*)(sQ + slab_off(t, i, 64)));
-                    }
-                    *(uint4*)(sPT + i * 128 + ((((c0 + j8) >> 3) ^ (i & 7)) << 4)) =
-                        make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
+                for (int t = 0; t < 64; t += 2) {
+                    const uint32_t lo = *(const uint16_t*)(qcol + t * 128 + ((ci ^ (t & 7)) << 4));
+                    const uint32_t hi = *(const uint16_t*)(qcol + (t + 1) * 128 + ((ci ^ ((t + 1) & 7)) << 4));
+                    qreg[t >> 1] = lo | (hi << 16);
                 }
             }
-            float* oi = (float*)(slot + SLOT_OI) + i;
+            mbar_arrive(&bar[B_QCOPIED]);
+            PF_LAP(20);
+            bool ok = PF_WAIT(B_SLOTOK, k & 1, 121);      // the ring slot may be written
+            ok = ok && PF_WAIT(B_D34DONE, k & 1, 123);
+            tc_fence_after();
+            if (!ok) return;
+            PF_LAP(21);
+            // ---- [E | Xi] from RA -> staging (E over W, Xi over Uh), bulk-stored by the store warp
+            {
+                uint8_t* sE = smem + b * F_REGION;
+                uint8_t* sXi = smem + b * F_REGION + F_STAGE_XI;
+#pragma unroll 1
+                for (int c0 = 0; c0 < DK + DV; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RA + lane_base + c0, rr);
+                    tmem_ld_wait();
+                    uint8_t* dst = (c0 < DK) ? sE : sXi;
+                    const int col8 = ((c0 < DK) ? c0 : c0 - DK) >> 3;
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(RB + lane_base + 64 + c0, rr);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (c0 + j < Cv) oi[(c0 + j) * DV] = __uint_as_float(rr[j]);
-            }
-            tc_fence_before();
-            mbar_arrive(&bar[B_D4FREE]);
-            // [E | Xi] from RA -> staging (E over W, Xi over Uh)
-#pragma unroll 2
-            for (int c0 = 0; c0 < DK + DV; c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(RA + lane_base + c0, rr);
-                tmem_ld_wait();
-                uint8_t* dst = (c0 < DK) ? sE : sXi;
-                const int col0 = (c0 < DK) ? c0 : c0 - DK;
-#pragma unroll
-                for (int j8 = 0; j8 < 32; j8 += 8) *(uint4*)(dst + slab_off(i, col0 + j8, 128)) = pack8(rr + j8, 1.f);
+                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + chunk_off(i, col8 + j8, 128)) = pack8(rr + 8 * j8, 1.f);
+                }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
             fence_async_smem();
-            named_bar(3, 128);
-            if (i == 0) {
-                bulk_store(slot + SLOT_E, sE, DK * DK * 2);
-                bulk_store(slot + SLOT_XI, sXi, DK * DV * 2);
-                bulk_store(slot + SLOT_QT, sPT, DK * 128);
-                bulk_commit();
-                bulk_wait_read_all();
-                mbar_arrive(&bar[B_XFREE + b]);
-                mbar_arrive(&bar[B_VFREE + b]);
-                mbar_arrive(&bar[B_PTFREE]);
-                bulk_wait_all();
-                fence_async_global();
-                __threadfence();
-                st_release_gpu(&ws.ready[seq * g.R + slot_i], c + 1);
+            mbar_arrive(&bar[B_STAGED]);
+            PF_LAP(22);
+            // ---- Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t]: row i of the Qt image, straight into the ring
+            {
+                uint8_t* qrow = slot + SLOT_QT + i * 128;
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RB + lane_base + c0, rr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t qq = qreg[(c0 >> 1) + 4 * j8 + j];
+                            const float2 qf = __half22float2(*reinterpret_cast<const __half2*>(&qq));
+                            w4[j] = pack_h2(__uint_as_float(rr[8 * j8 + 2 * j]) + qf.x, __uint_as_float(rr[8 * j8 + 2 * j + 1]) + qf.y);
+                        }
+                        *(uint4*)(qrow + (((((c0 >> 3) + j8)) ^ (i & 7)) << 4)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    }
+                }
             }
+            // ---- OI^T[j][t] -> OI[t][j] (fp32), straight into the ring
+            {
+                float* oi = (float*)(slot + SLOT_OI) + i;
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RB + lane_base + 64 + c0, rr);
+                    tmem_ld_wait();
+                    const int lim = Cv - c0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < lim) oi[(c0 + j) * DV] = __uint_as_float(rr[j]);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&bar[B_D4FREE]);
+            mbar_arrive(&bar[B_OUTDONE]);
+            PF_LAP(23);
         }
     } else if (warp == 12) {
         // ------------------------------------------------ TMA loads -------------------------------------------
         if (lane == 0) {
-            for (int j = 0; j <= nk; ++j) {
+#pragma unroll 1
+            for (int j = 0; j < nk; ++j) {
                 const int b = j & 1;
-                int seq = 0, c = 0;
-                if (j < nk) {
-                    item(j, seq, c);
-                    if (j >= 2 && !mbar_wait_clk(&bar[B_D34DONE], (j - 2) & 1, err, 131)) return;
-                    mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_3d(smem + F_K + b * 32768 + h * KV_SLAB, &maps.k, 64 * h, c * C * r, seq, &bar[B_KFULL + b]);
+                int seq, c;
+                item(j, seq, c);
+                // K: its region was last read by MMA3 of chunk j-2 (n = 64: and held part of that chunk's Xi image)
+                if (j >= 2 && !PF_WAIT(B_D34DONE, (j - 2) & 1, 131)) return;
+                if (N == 64 && j >= 2 && !PF_WAIT(B_VFREE + b, ((j >> 1) - 1) & 1, 134)) return;
+                mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
+                for (int h = 0; h < 2; ++h)
+                    tma_load_3d(smem + b * F_REGION + K_OFF + h * KV_SLAB, &maps.k, 64 * h, c * C * r, seq, &bar[B_KFULL + b]);
+                // Q: single buffer, free once P0^T of chunk j-1 is complete and the out warps hold their copy
+                if (j >= 1 && (!PF_WAIT(B_P0DONE, (j - 1) & 1, 132) || !PF_WAIT(B_QCOPIED, (j - 1) & 1, 136))) return;
+                mbar_expect_tx(&bar[B_QFULL], (uint32_t)C * 256);
+                for (int h = 0; h < 2; ++h) tma_load_3d(smem + F_Q + h * 8192, &maps.q, 64 * h, c * C, seq, &bar[B_QFULL]);
+                // V: its region holds the Xi image of chunk j-2 until the bulk store has read it
+                if (j >= 2 && !PF_WAIT(B_VFREE + b, ((j >> 1) - 1) & 1, 133)) return;
+                if (N == 64 && j >= 2 && !PF_WAIT(B_XFREE + b, ((j >> 1) - 1) & 1, 135)) return;
+                mbar_expect_tx(&bar[B_VFULL + b], K_BYTES);
+                for (int h = 0; h < 2; ++h)
+                    tma_load_3d(smem + b * F_REGION + V_OFF + h * KV_SLAB, &maps.v, 64 * h, c * C * r, seq, &bar[B_VFULL + b]);
+            }
+        }
+    } else if (warp == 13) {
+        // ------------------------------------------------ MMA issue (whole warp, converged) --------------------
+        if (nk > 0) {
+            const uint32_t q_b = smem_u32(smem + F_Q), pt_b = smem_u32(smem + F_PT);
+            if (!PF_WAIT(B_KFULL + 0, 0, 141)) return;
+            tc_fence_after();
+            {
+                const uint32_t k_b = smem_u32(smem + K_OFF);
+                gemm_uni<false, false, N, DK, N, N, true>(RB, k_b, k_b);     // G(0) = K K^T from the bf16 tile
+                commit_uni(&bar[B_GDONE]);
+            }
+#pragma unroll 1
+            for (int k = 0; k < nk; ++k) {
+                const int b = k & 1, b1 = b ^ 1;
+                const uint32_t x_b = smem_u32(smem + b * F_REGION + X_OFF), v_b = x_b + V_OFF, k_b = x_b + K_OFF;
+                // [Uh | W] (before the row scaling) = X [V | K]
+                if (!PF_WAIT(B_XREADY + b, (k >> 1) & 1, 142) || !PF_WAIT(B_V16 + b, (k >> 1) & 1, 143) ||
+                    !PF_WAIT(B_K16 + b, (k >> 1) & 1, 140))
+                    return;
+                if (k >= 1 && !PF_WAIT(B_RAFREE, (k - 1) & 1, 144)) return;
+                tc_fence_after();
+                gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
+                commit_uni(&bar[B_D2DONE]);
+                PF_LAP(30);
+                // P0^T = K Q^T   (RC was drained before MMA4 of chunk k-1 was issued)
+                if (!PF_WAIT(B_Q16, k & 1, 148)) return;
+                tc_fence_after();
+                gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
+                commit_uni(&bar[B_P0DONE]);
+                PF_LAP(32);
+                // G of the next chunk, from its bf16 tile
+                if (k + 1 < nk) {
+                    if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
+                    if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
+                    tc_fence_after();
+                    const uint32_t k1_b = smem_u32(smem + b1 * F_REGION + K_OFF);
+                    gemm_uni<false, false, N, DK, N, N, true>(RB, k1_b, k1_b);
+                    commit_uni(&bar[B_GDONE]);
                 }
-                if (j >= 1) {
-                    int sq, cq;
-                    item(j - 1, sq, cq);
-                    if (j >= 2 && !mbar_wait_clk(&bar[B_D4FREE], (j - 2) & 1, err, 132)) return;
-                    mbar_expect_tx(&bar[B_QFULL], (uint32_t)C * 256);
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_3d(smem + F_Q + h * 8192, &maps.q, 64 * h, cq * C, sq, &bar[B_QFULL]);
-                }
-                if (j < nk) {
-                    if (j >= 2 && !mbar_wait_clk(&bar[B_VFREE + b], ((j >> 1) - 1) & 1, err, 133)) return;
-                    mbar_expect_tx(&bar[B_VFULL + b], K_BYTES);
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_3d(smem + F_V + b * 32768 + h * KV_SLAB, &maps.v, 64 * h, c * C * r, seq, &bar[B_VFULL + b]);
-                }
+                PF_LAP(31);
+                // [E | Xi] = K^T [-W | Uh]
+                if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
+                tc_fence_after();
+                gemm_uni<true, true, DK + DV, N, N, N>(RA, k_b, x_b);
+                PF_LAP(33);
+                // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T   (RB: G of chunk k+1 must have been drained)
+                if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
+                if (k + 1 < nk && !PF_WAIT(B_GFREE, (k + 1) & 1, 151)) return;
+                tc_fence_after();
+                gemm_uni<true, true, 64, N, N, N>(RB, x_b, pt_b);
+                gemm_uni<true, true, 64, N, N, N>(RB + 64, v_b, pt_b);
+                commit_uni(&bar[B_D34DONE]);
+                PF_LAP(34);
             }
         }
     } else {
-        // ------------------------------------------------ MMA issue -------------------------------------------
-        if (lane == 0 && nk > 0) {
-            const uint32_t q_b = smem_u32(smem + F_Q), pt_b = smem_u32(smem + F_PT);
-            if (!mbar_wait_clk(&bar[B_K16 + 0], 0, err, 141)) return;
-            tc_fence_after();
-            {
-                const uint32_t k_b = smem_u32(smem + F_K);
-                gemm_issue<false, false>(RB, k_b, N, k_b, N, N, DK, false, false);     // G(0) = K K^T
-                mma_commit(&bar[B_GDONE]);
-            }
+        // ------------------------------------------------ store warp: staging -> ring, flags -----------------
+        if (lane == 0) {
+#pragma unroll 1
             for (int k = 0; k < nk; ++k) {
-                const int b = k & 1, b1 = b ^ 1;
-                const uint32_t k_b = smem_u32(smem + F_K + b * 32768), v_b = smem_u32(smem + F_V + b * 32768),
-                               x_b = smem_u32(smem + F_X + b * 32768);
-                // [W | Uh] = X [K | V]
-                if (!mbar_wait_clk(&bar[B_XREADY + b], (k >> 1) & 1, err, 142)) return;
-                if (!mbar_wait_clk(&bar[B_V16 + b], (k >> 1) & 1, err, 143)) return;
-                if (k >= 1 && !mbar_wait_clk(&bar[B_RAFREE], (k - 1) & 1, err, 144)) return;
-                tc_fence_after();
-                gemm_issue<false, true>(RA, x_b, N, k_b, N, DK, N, false, false);
-                gemm_issue<false, true>(RA + DK, x_b, N, v_b, N, DV, N, false, false);
-                mma_commit(&bar[B_D2DONE]);
-                // G of the next chunk
-                if (k + 1 < nk) {
-                    if (!mbar_wait_clk(&bar[B_K16 + b1], ((k + 1) >> 1) & 1, err, 145)) return;
-                    if (!mbar_wait_clk(&bar[B_GFREE], k & 1, err, 146)) return;
-                    if (k >= 1 && !mbar_wait_clk(&bar[B_D4FREE], (k - 1) & 1, err, 147)) return;
-                    tc_fence_after();
-                    const uint32_t k1_b = smem_u32(smem + F_K + b1 * 32768);
-                    gemm_issue<false, false>(RB, k1_b, N, k1_b, N, N, DK, false, false);
-                    mma_commit(&bar[B_GDONE]);
-                }
-                // P0^T = K Q^T
-                if (!mbar_wait_clk(&bar[B_Q16], k & 1, err, 148)) return;
-                tc_fence_after();
-                gemm_issue<false, false>(RC, k_b, N, q_b, 64, 64, DK, false, false);
-                mma_commit(&bar[B_P0DONE]);
-                // [E | Xi] = K^T [-W | Uh]
-                if (!mbar_wait_clk(&bar[B_WUREADY], k & 1, err, 149)) return;
-                tc_fence_after();
-                gemm_issue<true, true>(RA, k_b, N, x_b, N, DK, N, true, false);
-                gemm_issue<true, true>(RA + DK, k_b, N, v_b, N, DV, N, false, false);
-                // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T
-                if (!mbar_wait_clk(&bar[B_PTREADY], k & 1, err, 150)) return;
-                if (k + 1 < nk && !mbar_wait_clk(&bar[B_GFREE], (k + 1) & 1, err, 151)) return;
-                tc_fence_after();
-                gemm_issue<true, true>(RB, x_b, N, pt_b, N, 64, N, true, false);
-                gemm_issue<true, true>(RB + 64, v_b, N, pt_b, N, 64, N, false, false);
-                mma_commit(&bar[B_D34DONE]);
+                const int b = k & 1;
+                int seq, c;
+                item(k, seq, c);
+                const int slot_i = c % g.R;
+                uint8_t* slot = ws.ring + ((size_t)seq * g.R + slot_i) * SLOT_BYTES;
+                // the scan must be done with the chunk that used this slot before
+                if (c >= g.R && !flag_wait_ge(&ws.consumed[seq], c - g.R + 1, err, 161)) return;
+                mbar_arrive(&bar[B_SLOTOK]);
+                PF_LAP(60);
+                if (!PF_WAIT(B_STAGED, k & 1, 162)) return;
+                PF_LAP(61);
+                bulk_store(slot + SLOT_E, smem + b * F_REGION, DK * DK * 2);
+                bulk_store(slot + SLOT_XI, smem + b * F_REGION + F_STAGE_XI, DK * DV * 2);
+                bulk_commit();
+                bulk_wait_read_all();
+                mbar_arrive(&bar[B_XFREE + b]);
+                mbar_arrive(&bar[B_VFREE + b]);
+                PF_LAP(62);
+                bulk_wait_all();
+                if (!PF_WAIT(B_OUTDONE, k & 1, 163)) return;
+                fence_async_global();
+                __threadfence();
+                st_release_gpu(&ws.ready[seq * g.R + slot_i], c + 1);
+                PF_LAP(63);
             }
         }
     }
+    if (tim) atomicAdd(tim + 240 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));   // whole role, per warp
 }
 
 // =============================================================================================================
@@ -589,9 +710,14 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = g.NC;
     int* err = ws.status;
+    unsigned long long* const tim = timing_slot(ws, seq == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416));
+    const long long t_role = clock64();
+    long long t_lap = t_role;
+    (void)t_lap;
     const uint32_t t_delta = tb, t_o = tb + 128;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
+    const int* ready = ws.ready + seq * g.R;
 
     if (warp < 8) {
         // ------------------------------------------------ chain: the state lives here -------------------------
@@ -603,15 +729,13 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             float4 v4 = S0 ? *(const float4*)(S0 + srow + j) : make_float4(0.f, 0.f, 0.f, 0.f);
             S[j] = v4.x; S[j + 1] = v4.y; S[j + 2] = v4.z; S[j + 3] = v4.w;
         }
+#pragma unroll 1
         for (int c = 0; c < NC; ++c) {
-            const int st = c % SCAN_STAGES, buf = c & 1;
-            if (!mbar_wait_clk(&bar[B_FULL + st], (c / SCAN_STAGES) & 1, err, 201)) return;
-            // Xi row i, columns 64w..64w+63 (swizzled 16-byte chunks)
-            const uint8_t* xrow = ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_XI + w * 16384 + i * 128;
-            uint4 xi[8];
-#pragma unroll
-            for (int p = 0; p < 8; ++p) xi[p] = ld_cg_u4(xrow + ((p ^ (i & 7)) << 4));
+            const int buf = c & 1;
             // fp16 copy of the state: B operand of Delta, A operand of O^T
+            bool ok = true;
+            if (c >= 2) ok = PF_WAIT(B_S16FREE + buf, ((c >> 1) - 1) & 1, 201);
+            PF_LAP(40);
             uint8_t* sb = smem + S_S16 + buf * 32768 + w * 16384 + i * 128;
 #pragma unroll
             for (int p = 0; p < 8; ++p)
@@ -620,101 +744,141 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                                pack_h2(S[8 * p + 4], S[8 * p + 5]), pack_h2(S[8 * p + 6], S[8 * p + 7]));
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(&bar[B_SREADY + buf * 2 + w]);
-            if (!mbar_wait_clk(&bar[B_DDONE + w], c & 1, err, 202)) return;
+            mbar_arrive(&bar[B_SREADY + buf]);
+            if (!named_bar_and(1 + w, 128, ok)) return;
+            PF_LAP(41);
+            // this half's Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j], issued by the half's first warp
+            if ((warp & 3) == 0) {
+                if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
+                tc_fence_after();
+                gemm_uni<false, true, 64, DK, 128, 128>(t_delta + 64 * w, smem_u32(smem + S_E + buf * 32768),
+                                                        smem_u32(smem + S_S16 + buf * 32768 + w * 16384));
+                commit_uni(&bar[B_DDONE + w]);
+                commit_uni(&bar[B_EEMPTY + buf]);
+            }
+            if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
+            if (!PF_WAIT(B_DDONE + w, c & 1, 202)) return;
             tc_fence_after();
+            PF_LAP(42);
+            // S^T += Delta^T + Xi   (row i, columns 64w..64w+63; Xi from its swizzled image)
+            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + i * 128;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(t_delta + lane_base + 64 * w + c0, rr);
+                uint4 xi[4];
+#pragma unroll
+                for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((((c0 >> 3) + p) ^ (i & 7)) << 4));
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const uint32_t wd = ((const uint32_t*)&xi[(c0 + j) >> 3])[((c0 + j) & 7) >> 1];
+                    const uint32_t wd = ((const uint32_t*)&xi[j >> 3])[(j & 7) >> 1];
                     const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&wd));
                     S[c0 + j] += __uint_as_float(rr[j]) + xv.x;
                     S[c0 + j + 1] += __uint_as_float(rr[j + 1]) + xv.y;
                 }
             }
+            tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bar[B_EMPTY + st]);
+            if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
+            PF_LAP(43);
         }
         if (S_final)
 #pragma unroll
             for (int j = 0; j < 64; j += 4) *(float4*)(S_final + srow + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
     } else if (warp < 12) {
         // ------------------------------------------------ output: O^T = OI^T + S Qt^T --------------------------
+        // OI of the next chunk is fetched (into registers) while this chunk's MMA is awaited.
         const int j = tid - 256;
-        for (int c = 0; c < NC; ++c) {
-            const int st = c % SCAN_STAGES, ob = c & 1;
+        float a[64];
+        auto fetch_oi = [&](int c) -> bool {
+            int ok = 1;
+            if (lane == 0) ok = flag_wait_ge(&ready[c % g.R], c + 1, err, 211) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) return false;
             const int Cv = min(g.C, g.L - c * g.C);
-            if (!mbar_wait_clk(&bar[B_FULL + st], (c / SCAN_STAGES) & 1, err, 211)) return;
             const float* oi = (const float*)(ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_OI) + j;
+#pragma unroll
+            for (int t = 0; t < 64; ++t) a[t] = (t < Cv) ? ld_cg_f32(oi + t * DV) : 0.f;
+            return true;
+        };
+#pragma unroll 1
+        for (int c = 0; c < NC; ++c) {
+            const int ob = c & 1;
+            const int Cv = min(g.C, g.L - c * g.C);
+            if (c == 0 && !fetch_oi(0)) return;
             float* orow = O + ((long long)seq * g.L + (long long)c * g.C) * DV + j;
+            if (!PF_WAIT(B_ODONE + ob, (c >> 1) & 1, 212)) return;
+            tc_fence_after();
+            PF_LAP(45);
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
-                float a[32];
-#pragma unroll
-                for (int t = 0; t < 32; ++t) a[t] = (c0 + t < Cv) ? ld_cg_f32(oi + (c0 + t) * DV) : 0.f;
-                if (c0 == 0) {
-                    if (!mbar_wait_clk(&bar[B_ODONE + ob], (c >> 1) & 1, err, 212)) return;
-                    tc_fence_after();
-                }
                 uint32_t rr[32];
                 tmem_ld32(t_o + ob * 64 + lane_base + c0, rr);
                 tmem_ld_wait();
 #pragma unroll
                 for (int t = 0; t < 32; ++t)
-                    if (c0 + t < Cv) orow[(long long)(c0 + t) * DV] = a[t] + __uint_as_float(rr[t]);
+                    if (c0 + t < Cv) orow[(long long)(c0 + t) * DV] = a[c0 + t] + __uint_as_float(rr[t]);
             }
             tc_fence_before();
             mbar_arrive(&bar[B_OFREE + ob]);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar[B_EMPTY + st]);
+            PF_LAP(46);
+            if (c + 1 < NC && !fetch_oi(c + 1)) return;
+            PF_LAP(47);
         }
     } else if (warp == 12) {
         // ------------------------------------------------ producer: ring -> shared memory ----------------------
         if (lane == 0) {
-            for (int c = 0; c < NC; ++c) {
-                const int st = c % SCAN_STAGES;
-                if (c >= SCAN_STAGES) {
-                    if (!mbar_wait_clk(&bar[B_EMPTY + st], ((c / SCAN_STAGES) - 1) & 1, err, 221)) return;
-                    st_release_gpu(&ws.consumed[seq], c - SCAN_STAGES + 1);
-                }
-                const int slot_i = c % g.R;
-                if (!flag_wait_ge(&ws.ready[seq * g.R + slot_i], c + 1, err, 222)) return;
+            auto load_e = [&](int c) -> bool {
+                const int st = c & 1;
+                if (!flag_wait_ge(&ready[c % g.R], c + 1, err, 222)) return false;
                 fence_async_global();
-                const uint8_t* slot = ring + (size_t)slot_i * SLOT_BYTES;
-                uint8_t* dst = smem + S_STAGE + st * S_STAGE_BYTES;
-                mbar_expect_tx(&bar[B_FULL + st], DK * DK * 2 + DK * 128);
-                bulk_load(dst, slot + SLOT_E, DK * DK * 2, &bar[B_FULL + st]);
-                bulk_load(dst + 32768, slot + SLOT_QT, DK * 128, &bar[B_FULL + st]);
+                if (c >= 2 && !PF_WAIT(B_EEMPTY + st, ((c >> 1) - 1) & 1, 221)) return false;
+                mbar_expect_tx(&bar[B_EFULL + st], DK * DK * 2);
+                bulk_load(smem + S_E + st * 32768, ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_E, DK * DK * 2, &bar[B_EFULL + st]);
+                return true;
+            };
+#pragma unroll 1
+            for (int c = 0; c < NC; ++c) {
+                if (c == 0 && !load_e(0)) return;
+                // (the flag of chunk c was acquired by load_e(c))
+                const uint8_t* slot = ring + (size_t)(c % g.R) * SLOT_BYTES;
+                const int b = c & 1;
+                if (c >= 2 && !PF_WAIT(B_XIEMPTY + b, ((c >> 1) - 1) & 1, 224)) return;
+                mbar_expect_tx(&bar[B_XIFULL + b], DK * DV * 2);
+                bulk_load(smem + S_XI + b * 32768, slot + SLOT_XI, DK * DV * 2, &bar[B_XIFULL + b]);
+                if (c >= 2 && !PF_WAIT(B_QTEMPTY + b, ((c >> 1) - 1) & 1, 223)) return;
+                mbar_expect_tx(&bar[B_QTFULL + b], DK * 128);
+                bulk_load(smem + S_QT + b * 16384, slot + SLOT_QT, DK * 128, &bar[B_QTFULL + b]);
+                PF_LAP(50);
+                if (c + 1 < NC && !load_e(c + 1)) return;
+                PF_LAP(51);
             }
         }
-    } else {
-        // ------------------------------------------------ MMA issue -------------------------------------------
-        if (lane == 0) {
-            for (int c = 0; c < NC; ++c) {
-                const int st = c % SCAN_STAGES, buf = c & 1, ob = c & 1;
-                const uint32_t e_b = smem_u32(smem + S_STAGE + st * S_STAGE_BYTES), qt_b = e_b + 32768;
-                const uint32_t s_b = smem_u32(smem + S_S16 + buf * 32768);
-                if (!mbar_wait_clk(&bar[B_FULL + st], (c / SCAN_STAGES) & 1, err, 231)) return;
-                for (int w = 0; w < 2; ++w) {
-                    if (!mbar_wait_clk(&bar[B_SREADY + buf * 2 + w], (c >> 1) & 1, err, 232)) return;
-                    tc_fence_after();
-                    // Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j],  j in the half w
-                    gemm_issue<false, true>(t_delta + 64 * w, e_b, 128, s_b + w * 16384, 128, 64, DK, false, false);
-                    mma_commit(&bar[B_DDONE + w]);
-                }
-                if (c >= 2 && !mbar_wait_clk(&bar[B_OFREE + ob], ((c >> 1) - 1) & 1, err, 233)) return;
-                tc_fence_after();
-                // O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
-                gemm_issue<true, true>(t_o + ob * 64, s_b, 128, qt_b, 128, 64, DK, false, false);
-                mma_commit(&bar[B_ODONE + ob]);
-                mma_commit(&bar[B_EMPTY + st]);
-            }
+    } else if (warp == 13) {
+        // ------------------------------------------------ O^T MMA issue (whole warp), consumed reports --------
+#pragma unroll 1
+        for (int c = 0; c < NC; ++c) {
+            const int buf = c & 1, ob = c & 1;
+            PF_LAP(70);
+            if (!PF_WAIT(B_SREADY + buf, (c >> 1) & 1, 232) || !PF_WAIT(B_QTFULL + ob, (c >> 1) & 1, 234)) return;
+            if (c >= 2 && !PF_WAIT(B_OFREE + ob, ((c >> 1) - 1) & 1, 233)) return;
+            tc_fence_after();
+            PF_LAP(71);
+            // O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
+            gemm_uni<true, true, 64, DK, 128, 128>(t_o + ob * 64, smem_u32(smem + S_S16 + buf * 32768), smem_u32(smem + S_QT + ob * 16384));
+            commit_uni(&bar[B_ODONE + ob]);
+            commit_uni(&bar[B_QTEMPTY + ob]);
+            commit_uni(&bar[B_S16FREE + buf]);
+            PF_LAP(72);
+            // the output warps are done with chunk c-2, hence the chain with chunk c-3: chunks < c-2 are
+            // consumed and their ring slots may be rewritten
+            if (c >= 2 && lane == 0) st_release_gpu(&ws.consumed[seq], c - 2);
+            __syncwarp();
+            PF_LAP(73);
         }
     }
+    if (tim) atomicAdd(tim + 260 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));   // whole role, per warp
 }
 
 template <int N>
@@ -733,9 +897,13 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     }
     if (tid == 0) {
         if (is_scan) {
-            for (int s = 0; s < SCAN_STAGES; ++s) { mbar_init(&bar[B_FULL + s], 1); mbar_init(&bar[B_EMPTY + s], 13); }
-            for (int x = 0; x < 4; ++x) mbar_init(&bar[B_SREADY + x], 128);
-            for (int x = 0; x < 2; ++x) { mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128); }
+            for (int x = 0; x < 2; ++x) {
+                mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 2);
+                mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
+                mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
+                mbar_init(&bar[B_SREADY + x], 256); mbar_init(&bar[B_S16FREE + x], 1);
+                mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
+            }
         } else {
             for (int x = 0; x < 2; ++x) {
                 mbar_init(&bar[B_KFULL + x], 1); mbar_init(&bar[B_VFULL + x], 1);
@@ -748,7 +916,8 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
             mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 128);
             mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 128);
             mbar_init(&bar[B_D34DONE], 1); mbar_init(&bar[B_D4FREE], 128); mbar_init(&bar[B_RAFREE], 128);
-            mbar_init(&bar[B_PTFREE], 1);
+            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_STAGED], 128); mbar_init(&bar[B_OUTDONE], 128);
+            mbar_init(&bar[B_SLOTOK], 1);
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.v);
@@ -768,6 +937,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
 
     if (is_scan) scan_role(g, ws, S0, O, S_final, smem, bar, tb, (int)blockIdx.x);
     else flow_role<N>(maps, g, ws, beta, smem, bar, tb, (int)blockIdx.x - g.n_scan);
+
 
     tc_fence_before();
     __syncthreads();
@@ -813,9 +983,11 @@ int sm_count() {
     return sms;
 }
 
+int g_ring_depth = 8;     // slots per sequence (option "ring_depth", 3..64)
+
 int ring_depth(const Problem& p) {
     const int NC = p.chunks_per_seq();
-    return NC < 8 ? (NC < 1 ? 1 : NC) : 8;
+    return NC < g_ring_depth ? (NC < 1 ? 1 : NC) : g_ring_depth;
 }
 
 struct Carve {
@@ -826,7 +998,7 @@ Carve carve(const Problem& p) {
     const int R = ring_depth(p);
     Carve c{};
     c.status = 0;
-    c.ready = 1024;
+    c.ready = 4096;
     c.consumed = c.ready + align_up(nseq * R * 4, 256);
     c.flag_bytes = align_up(c.consumed + nseq * 4, 1024);
     c.ring = c.flag_bytes;
@@ -835,6 +1007,15 @@ Carve carve(const Problem& p) {
 }
 
 }  // namespace
+
+int fused_set_option(const char* name, int value) {
+    if (strcmp(name, "ring_depth") == 0) {
+        if (value < 3 || value > 64) return PF_ERR_INVALID;
+        g_ring_depth = value;
+        return PF_OK;
+    }
+    return PF_ERR_UNSUPPORTED;
+}
 
 bool fused_supported(const Problem& p) {
     if (p.in_dtype != PF_DTYPE_BF16 || p.d_k != DK || p.d_v != DV) return false;

@@ -64,11 +64,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* e
 // the waits of the fused kernel sit on latency-critical paths.  Also gives up early once another
 // thread has reported a failure in *err_flag, so that one expired wait drains the whole grid quickly.
 constexpr long long WAIT_CYCLES = 2000000000ll;
-__device__ __forceinline__ bool mbar_wait_clk(uint64_t* bar, uint32_t parity, int* err_flag, int code) {
-    if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is kept out of line: dozens of call sites would otherwise bloat the instruction footprint.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, int* err_flag, int code) {
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar_addr), "r"(parity)
+            : "memory");
+        if (ok) return true;
         if ((it & 255u) == 0) {
             if (clock64() - t0 > WAIT_CYCLES) break;
             if ((it & 4095u) == 0 && *(volatile int*)err_flag != 0) return false;
@@ -76,6 +82,18 @@ __device__ __forceinline__ bool mbar_wait_clk(uint64_t* bar, uint32_t parity, in
     }
     atomicCAS(err_flag, 0, code);
     return false;
+}
+// `tim` (diagnostic builds only, else null): per-code accumulators of the cycles spent waiting.
+__device__ __forceinline__ bool mbar_wait_clk(uint64_t* bar, uint32_t parity, int* err_flag, int code,
+                                              unsigned long long* tim = nullptr) {
+    if (tim) {      // (one try_wait may itself block for a while before it reports)
+        const long long t0 = clock64();
+        const bool ok = mbar_try_wait(bar, parity) || mbar_wait_slow(smem_u32(bar), parity, err_flag, code);
+        atomicAdd(tim + code, (unsigned long long)(clock64() - t0));
+        return ok;
+    }
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(smem_u32(bar), parity, err_flag, code);
 }
 
 // ---- named barriers, global-memory flags, cache-bypassing loads ----------------------------------------
@@ -113,7 +131,7 @@ __device__ __forceinline__ float ld_cg_f32(const float* p) {
     return v;
 }
 // Waits until *p >= want (acquire), bounded by elapsed cycles.
-__device__ __forceinline__ bool flag_wait_ge(const int* p, int want, int* err_flag, int code) {
+static __device__ __noinline__ bool flag_wait_ge(const int* p, int want, int* err_flag, int code) {
     if (ld_acquire_gpu(p) >= want) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
@@ -241,6 +259,33 @@ __device__ __forceinline__ void gemm_issue(uint32_t d_tmem, uint32_t a_base, int
         else bd = desc_kmajor(b_base + (uint32_t)(kk >> 2) * (uint32_t)b_rows * 128u + (uint32_t)(kk & 3) * 32u);
         mma_f16(d_tmem, ad, bd, idesc, accumulate_first || kk > 0);
     }
+}
+
+// Warp-uniform issue with every shape known at compile time: the WHOLE warp runs this (converged) and one
+// elected lane issues each instruction.  The two base descriptors are built once and each K-step only adds a
+// constant to the start-address field; with uniform control flow that arithmetic stays in the uniform
+// datapath, which makes the issue several times cheaper than a single diverged lane rebuilding descriptors.
+// BF16: both operands are bf16 instead of fp16 (same 16-bit layouts).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
+__device__ __forceinline__ void gemm_uni(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
+    constexpr uint32_t idesc = make_idesc(NCOLS, A_MN, B_MN, false) | (BF16 ? ((1u << 7) | (1u << 10)) : 0u);
+    const uint64_t a0 = A_MN ? desc_mnmajor(a_base, (uint32_t)A_ROWS * 128u) : desc_kmajor(a_base);
+    const uint64_t b0 = B_MN ? desc_mnmajor(b_base, (uint32_t)B_ROWS * 128u) : desc_kmajor(b_base);
+#pragma unroll
+    for (int kk = 0; kk < KDIM / 16; ++kk) {
+        const uint32_t a_off = A_MN ? (uint32_t)kk * 2048u : (uint32_t)(kk >> 2) * (uint32_t)A_ROWS * 128u + (uint32_t)(kk & 3) * 32u;
+        const uint32_t b_off = B_MN ? (uint32_t)kk * 2048u : (uint32_t)(kk >> 2) * (uint32_t)B_ROWS * 128u + (uint32_t)(kk & 3) * 32u;
+        const uint64_t ad = a0 + (uint64_t)(a_off >> 4), bd = b0 + (uint64_t)(b_off >> 4);
+        if (elect_one()) mma_f16(d_tmem, ad, bd, idesc, kk > 0);
+    }
+}
+__device__ __forceinline__ void commit_uni(uint64_t* bar) {
+    if (elect_one()) mma_commit(bar);
 }
 
 // ---- warp-level MMA for the small triangular solve -------------------------------------------------
