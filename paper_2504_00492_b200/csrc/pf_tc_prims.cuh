@@ -216,6 +216,30 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
     return d;
 }
+// ---- unswizzled ("interleaved") operands ---------------------------------------------------------------
+// A matrix X[R rows][Cc cols] of 16-bit elements stored as Cc/8 column groups; group g holds columns 8g..8g+7
+// as R rows of 16 bytes:  offset(row, col) = (col/8)*R*16 + row*16 + (col%8)*2.  Eight consecutive rows of a
+// group are one 128-byte core matrix.  A warp whose lane l writes the 16-byte piece of row (r0 + l) writes
+// 512 contiguous bytes, which is why images that cross global memory use this form.
+//   K-major  (contraction index = column): core matrices 128 B apart along MN (SBO), R*16 apart along K (LBO)
+//   MN-major (contraction index = row)   : core matrices 128 B apart along K (LBO), R*16 apart along MN (SBO)
+__device__ __host__ __forceinline__ uint32_t ns_off(int row, int col, int R) {
+    return (uint32_t)(col >> 3) * (uint32_t)R * 16u + (uint32_t)row * 16u + ((uint32_t)col & 7u) * 2u;
+}
+__device__ __forceinline__ uint64_t make_desc_ns(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell); swizzle field 0 = none
+    return d;
+}
+__device__ __forceinline__ uint64_t desc_ns_kmajor(uint32_t saddr, int R) { return make_desc_ns(saddr, (uint32_t)R * 16u, 128u); }
+__device__ __forceinline__ uint64_t desc_ns_mnmajor(uint32_t saddr, int R) { return make_desc_ns(saddr, 128u, (uint32_t)R * 16u); }
+// byte advance of the start address per K-step of 16
+__device__ __host__ __forceinline__ uint32_t ns_kstep_kmajor(int R) { return 2u * (uint32_t)R * 16u; }
+__device__ __host__ constexpr uint32_t ns_kstep_mnmajor() { return 256u; }
+
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) { return make_desc(saddr, 16, 1024); }
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t slab_bytes) {
     return make_desc(saddr, slab_bytes, 1024);

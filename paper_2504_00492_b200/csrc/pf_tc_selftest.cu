@@ -19,22 +19,23 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
     __shared__ uint64_t bar;
     __shared__ uint32_t tmem_base;
     const bool a_mn = variant & 1, b_mn = variant & 2, neg = variant & 4;
+    const bool a_ns = variant & 8, b_ns = variant & 16;      // operand stored unswizzled (column groups of 8)
     const int tid = threadIdx.x, warp = tid >> 5;
 
     // A is given row-major as [128][128] in both cases: K-major -> A[m][k]; MN-major -> A[k][m].
     for (int e = tid; e < 128 * 128; e += 128) {
         const int row = e >> 7, col = e & 127;
-        *(__half*)(sA + slab_off(row, col, 128)) = A[e];
+        *(__half*)(sA + (a_ns ? ns_off(row, col, 128) : slab_off(row, col, 128))) = A[e];
     }
     if (!b_mn) {   // B[n][k]: N rows, 128 cols
         for (int e = tid; e < N * 128; e += 128) {
             const int row = e >> 7, col = e & 127;
-            *(__half*)(sB + slab_off(row, col, N)) = B[e];
+            *(__half*)(sB + (b_ns ? ns_off(row, col, N) : slab_off(row, col, N))) = B[e];
         }
     } else {       // B[k][n]: 128 rows, N cols
         for (int e = tid; e < 128 * N; e += 128) {
             const int row = e / N, col = e % N;
-            *(__half*)(sB + slab_off(row, col, 128)) = B[e];
+            *(__half*)(sB + (b_ns ? ns_off(row, col, 128) : slab_off(row, col, 128))) = B[e];
         }
     }
     if (tid == 0) {
@@ -52,7 +53,17 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
     if (tid == 0) {
         const uint32_t a_base = smem_u32(sA), b_base = smem_u32(sB);
         const int b_rows = b_mn ? 128 : N;
-        if (a_mn && b_mn) gemm_issue<true, true>(tb, a_base, 128, b_base, b_rows, N, 128, neg, false);
+        if (a_ns || b_ns) {
+            const uint32_t idesc = make_idesc(N, a_mn, b_mn, neg);
+            for (int kk = 0; kk < 8; ++kk) {
+                uint64_t ad, bd;
+                if (a_ns) ad = a_mn ? desc_ns_mnmajor(a_base + kk * ns_kstep_mnmajor(), 128) : desc_ns_kmajor(a_base + kk * ns_kstep_kmajor(128), 128);
+                else ad = a_mn ? desc_mnmajor(a_base + kk * 2048u, 128u * 128u) : desc_kmajor(a_base + (kk >> 2) * 128u * 128u + (kk & 3) * 32u);
+                if (b_ns) bd = b_mn ? desc_ns_mnmajor(b_base + kk * ns_kstep_mnmajor(), b_rows) : desc_ns_kmajor(b_base + kk * ns_kstep_kmajor(b_rows), b_rows);
+                else bd = b_mn ? desc_mnmajor(b_base + kk * 2048u, (uint32_t)b_rows * 128u) : desc_kmajor(b_base + (kk >> 2) * (uint32_t)b_rows * 128u + (kk & 3) * 32u);
+                mma_f16(tb, ad, bd, idesc, kk > 0);
+            }
+        } else if (a_mn && b_mn) gemm_issue<true, true>(tb, a_base, 128, b_base, b_rows, N, 128, neg, false);
         else if (a_mn) gemm_issue<true, false>(tb, a_base, 128, b_base, b_rows, N, 128, neg, false);
         else if (b_mn) gemm_issue<false, true>(tb, a_base, 128, b_base, b_rows, N, 128, neg, false);
         else gemm_issue<false, false>(tb, a_base, 128, b_base, b_rows, N, 128, neg, false);
@@ -80,7 +91,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
 extern "C" int pf_tc_selftest(int variant, const void* A, const void* B, float* D, int N, void* stream) {
     using namespace pf;
     if (!A || !B || !D) return PF_ERR_INVALID;
-    if (variant < 0 || variant > 7) return PF_ERR_INVALID;
+    if (variant < 0 || variant > 31) return PF_ERR_INVALID;
     if (N < 16 || N > 256 || (N % 16)) return PF_ERR_UNSUPPORTED;
     int dev = 0, major = 0;
     PF_CUDA_TRY(cudaGetDevice(&dev));

@@ -5,12 +5,12 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("variant", range(8))
+@pytest.mark.parametrize("variant", list(range(8)) + [8, 9, 16, 18, 24, 27, 10, 17])
 @pytest.mark.parametrize("N", [32, 64, 128, 192, 256])
 def test_tcgen05_gemm_variants(variant, N):
     from paper_2504_00492_b200 import binding
     g = torch.Generator().manual_seed(100 * variant + N)
-    a_mn, b_mn, neg = bool(variant & 1), bool(variant & 2), bool(variant & 4)
+    a_mn, b_mn, neg = bool(variant & 1), bool(variant & 2), bool(variant & 4)   # bits 3, 4: unswizzled staging
     A = (torch.randn(128, 128, generator=g) * 0.1).half()        # [m][k] or [k][m]
     Bm = (torch.randn(N, 128, generator=g) * 0.1).half()         # logical B[n][k]
     A_log = A.t() if a_mn else A                                  # logical A[m][k]
