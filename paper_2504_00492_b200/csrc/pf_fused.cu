@@ -20,17 +20,21 @@
 // A flow CTA is software-pipelined over two chunks (15 warps):
 //   warps 0-3  "solve"  epilogue of G = K K^T (mask, column scaling, fp16) and the triangular inverse
 //   warps 4-7  "mid"    epilogues of [Uh | W] and P^T; bf16 -> fp16 conversion of K, V, Q
-//   warps 8-11 "out"    epilogues of [E | Xi] (staged, bulk-stored) and [Qt^T | OI^T] (stored directly)
+//   warps 8-11 "out"    epilogues of [E | Xi] and [Qt^T | OI^T], stored straight into the ring
 //   warp 12             TMA loads (K and V double-buffered, Q single)
 //   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
-//   warp 14             bulk stores into the ring, ring back-pressure, ready flags
+//   warp 14             ring back-pressure and ready flags
 // Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi]; RB = [256,384) holds G of the NEXT
 // chunk and then [Qt^T | OI^T] of the current one; RC = [384,448) holds P0^T.
 // G is formed from the bf16 tiles as they land (both operands raw); every other product has a derived fp16
 // operand, so K, V and Q are converted to fp16 in place, off the critical path.
 //
-// A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns; the
-// first warp of each half issues that half's Delta MMAs), warps 8-11 add OI and write O, warp 12 streams
+// The images that cross the ring are laid out in unswizzled column groups (ns_off): a warp whose lanes hold
+// consecutive rows then writes 512 contiguous bytes per store, and the scan's bulk copies bring them into
+// shared memory in a form the MMA descriptors read directly.
+//
+// A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns; warp 0
+// issues the Delta MMA for both halves), warps 8-11 add OI and write O, warp 12 streams
 // the E / Xi / Qt images in with bulk copies, warp 13 issues the O^T MMAs and reports consumed chunks.
 //
 // Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
@@ -51,9 +55,9 @@ constexpr int FT = 480;                 // threads per CTA
 constexpr int DK = 128, DV = 128;
 
 // ---- ring slot layout (bytes) ---------------------------------------------------------------------------
-constexpr uint32_t SLOT_E = 0;                          // E image : fp16 [2 slabs][128 rows i][128 B]   (K-major A)
-constexpr uint32_t SLOT_QT = SLOT_E + DK * DK * 2;      // Qt image: fp16 [128 rows i][128 B = 64 t]     (MN-major B)
-constexpr uint32_t SLOT_XI = SLOT_QT + DK * 128;        // Xi image: fp16 [2 slabs (j half)][128 rows i][128 B]
+constexpr uint32_t SLOT_E = 0;                          // E image : fp16 [16 groups i'/8][128 rows i][16 B]  (K-major A)
+constexpr uint32_t SLOT_QT = SLOT_E + DK * DK * 2;      // Qt image: fp16 [ 8 groups t/8 ][128 rows i][16 B]  (MN-major B)
+constexpr uint32_t SLOT_XI = SLOT_QT + DK * 128;        // Xi image: fp16 [16 groups j/8 ][128 rows i][16 B]
 constexpr uint32_t SLOT_OI = SLOT_XI + DK * DV * 2;     // OI      : fp32 [64 rows t][128 cols j]
 constexpr uint32_t SLOT_BYTES = SLOT_OI + 64 * DV * 4;  // 114688
 
@@ -76,10 +80,8 @@ struct FusedMaps {
 
 // ---- shared memory ----------------------------------------------------------------------------------------
 // flow role: two 96 KB regions (chunk parity), each holding  X/W | V/Uh | K  back to back (n*256 bytes each),
-// so that [V | K] and [W | Uh] are single 256-column B operands.  After the chunk's last MMA the region is
-// staging space: the E image at +0, the Xi image at +32 KB.
+// so that [V | K] and [W | Uh] are single 256-column B operands.
 constexpr int F_REGION = 98304;
-constexpr int F_STAGE_XI = 32768;
 constexpr int F_Q = 2 * F_REGION;               // 16 KB      Q
 constexpr int F_PT = F_Q + 16384;               // 16 KB      P^T
 constexpr int F_BETA = F_PT + 16384;            // 2 x 128 fp32
@@ -112,22 +114,19 @@ enum {
     B_D34DONE = 18,   // mma: [E | Xi] and [Qt^T | OI^T] complete
     B_D4FREE = 19,    // out: RB drained
     B_RAFREE = 20,    // out: RA drained
-    B_XFREE = 21,     // [2] store warp: bulk store finished reading the E staging
-    B_VFREE = 23,     // [2] store warp: ... the Xi staging
     B_QCOPIED = 25,   // out: Q copied into registers
-    B_STAGED = 26,    // out: E and Xi images staged
-    B_OUTDONE = 27,   // out: Qt and OI stored
+    B_OUTDONE = 27,   // out: the chunk's images are stored
     B_SLOTOK = 28,    // store warp: the chunk's ring slot may be written
     // scan role
     B_EFULL = 32,     // [2] producer: E image landed
-    B_EEMPTY = 34,    // [2] chain: both Delta halves of that chunk complete (two commits)
+    B_EEMPTY = 34,    // [2] chain: Delta of that chunk complete
     B_XIFULL = 36,    // [2] producer: Xi image landed
     B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
     B_SREADY = 44,    // [2 buffers] chain: fp16 copy of the state published (256 arrivals)
     B_S16FREE = 46,   // [2 buffers] mma: the O^T MMA that reads the copy is complete
-    B_DDONE = 48,     // [2 halves] Delta half complete
+    B_DDONE = 48,     // Delta complete
     B_ODONE = 50,     // [2] mma: O^T complete
     B_OFREE = 52,     // [2] output warps: O^T drained
     B_COUNT = 54
@@ -145,19 +144,31 @@ __device__ __forceinline__ unsigned long long* timing_slot(const FusedWs& ws, bo
 #endif
 }
 #ifdef PF_TIMING
-#define PF_LAP(slot)                                                              \
-    do {                                                                          \
-        if (tim) {                                                                \
-            const long long n_ = clock64();                                       \
-            atomicAdd(tim + (slot), (unsigned long long)(n_ - t_lap));            \
-            t_lap = n_;                                                           \
-        }                                                                         \
+#define PF_LAP(id)                                          \
+    do {                                                    \
+        if (tim) {                                          \
+            const long long n_ = clock64();                 \
+            lapacc[(id)] += n_ - t_lap;                     \
+            t_lap = n_;                                     \
+        }                                                   \
+    } while (0)
+#define PF_LAP_FLUSH(role)                                                                              \
+    do {                                                                                                \
+        if (tim)                                                                                        \
+            for (int l_ = 0; l_ < 8; ++l_) atomicAdd(tim + 8 * (role) + l_, (unsigned long long)lapacc[l_]); \
     } while (0)
 #else
-#define PF_LAP(slot) do { } while (0)
+#define PF_LAP(id) do { } while (0)
+#define PF_LAP_FLUSH(role) do { } while (0)
 #endif
 
-#define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code, tim)
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+#define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code)
 
 // byte offset of the 16-byte chunk `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
 __device__ __forceinline__ uint32_t chunk_off(int row, int col8, int R) {
@@ -270,8 +281,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     unsigned long long* const tim =
         timing_slot(ws, fid == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416 || tid == 448));
     const long long t_role = clock64();
+    const unsigned long long t_ns = tim ? globaltimer_ns() : 0ull;
     long long t_lap = t_role;
-    (void)t_lap;
+    long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    (void)t_lap; (void)lapacc;
     const int nk = fid < g.items ? (g.items - fid + g.n_flow - 1) / g.n_flow : 0;
     const uint32_t RA = tb, RB = tb + 256, RC = tb + 384;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -314,12 +327,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
             bool ok = true;
-            if (k >= 2) ok = PF_WAIT(B_XFREE + b, ((k >> 1) - 1) & 1, 101);
-            sB[m] = bm;     // the readers of this half (chunk k-2) are done: X of chunk k-2 has been released
+            if (k >= 2) ok = PF_WAIT(B_D34DONE, (k - 2) & 1, 101);     // W of chunk k-2 (in this X region) has been read
+            sB[m] = bm;     // (the beta half of chunk k-2 was last read by that chunk's [Uh | W] epilogue)
             ok = ok && PF_WAIT(B_GDONE, k & 1, 102);
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
-            PF_LAP(1);
+            PF_LAP(0);
             // A = Mstrict (.) (G diag(beta)) as fp16 into X; column groups right of the warp's rows are zero
 #pragma unroll 1
             for (int c0 = 0; c0 < N; c0 += 32) {
@@ -348,7 +361,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_before();
             mbar_arrive(&bar[B_GFREE]);
             named_bar(1, 128);
-            PF_LAP(2);
+            PF_LAP(1);
             // 16x16 diagonal blocks: forward substitution, one thread per column of one block (fp32)
             float x[16];
             const int bk = tid >> 4, cc = tid & 15;
@@ -385,14 +398,15 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     *(__half*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4) + (cc & 7) * 2) = __float2half_rn(x[mm]);
             }
             named_bar(1, 128);
-            PF_LAP(3);
+            PF_LAP(2);
             merge_level<N, 16>(x_b, sX, warp, lane);
             merge_level<N, 32>(x_b, sX, warp, lane);
             if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
             fence_async_smem();
             mbar_arrive(&bar[B_XREADY + b]);
-            PF_LAP(4);
+            PF_LAP(3);
         }
+        PF_LAP_FLUSH(0);
     } else if (warp < 8) {
         // ------------------------------------------------ mid: [Uh | W] and P^T epilogues, conversions --------
         const int m = tid - 128;
@@ -423,7 +437,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // ---- RA = X [V | K]:  Uh = diag(beta) (X V) over V,  -W = -diag(beta) (X K) over X, fp16 operands
             if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
             tc_fence_after();
-            PF_LAP(12);
+            PF_LAP(0);
             {
                 const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
                 uint8_t* sU = smem + b * F_REGION + V_OFF;
@@ -445,11 +459,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_WUREADY]);
-            PF_LAP(13);
+            PF_LAP(1);
             // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
             if (k >= 1 && !PF_WAIT(B_D34DONE, (k - 1) & 1, 116)) return;
             if (!PF_WAIT(B_P0DONE, k & 1, 117)) return;
             tc_fence_after();
+            PF_LAP(2);
 #pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
@@ -472,29 +487,28 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_PTREADY]);
-            PF_LAP(11);
+            PF_LAP(3);
             // ---- conversions for chunk k+1 (K only once its Gram product has read the bf16 tile)
             if (k + 1 < nk) {
                 if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
-                PF_LAP(14);
+                PF_LAP(4);
                 cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
                 fence_async_smem();
                 mbar_arrive(&bar[B_K16 + b1]);
-                PF_LAP(15);
+                PF_LAP(5);
                 if (!PF_WAIT(B_QFULL, (k + 1) & 1, 114)) return;
-                PF_LAP(16);
                 cvt_region(smem + F_Q, 16384, m);
                 fence_async_smem();
                 mbar_arrive(&bar[B_Q16]);
-                PF_LAP(17);
+                PF_LAP(6);
                 if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
-                PF_LAP(18);
                 cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
                 fence_async_smem();
                 mbar_arrive(&bar[B_V16 + b1]);
-                PF_LAP(19);
+                PF_LAP(7);
             }
         }
+        PF_LAP_FLUSH(1);
     } else if (warp < 12) {
         // ------------------------------------------------ out: flow -> ring -----------------------------------
         const int i = tid - 256;
@@ -520,35 +534,32 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 }
             }
             mbar_arrive(&bar[B_QCOPIED]);
-            PF_LAP(20);
+            PF_LAP(0);
             bool ok = PF_WAIT(B_SLOTOK, k & 1, 121);      // the ring slot may be written
             ok = ok && PF_WAIT(B_D34DONE, k & 1, 123);
             tc_fence_after();
             if (!ok) return;
-            PF_LAP(21);
-            // ---- [E | Xi] from RA -> staging (E over W, Xi over Uh), bulk-stored by the store warp
+            PF_LAP(1);
+            // ---- [E | Xi] from RA: row i of both images, one 16-byte piece per column group
             {
-                uint8_t* sE = smem + b * F_REGION;
-                uint8_t* sXi = smem + b * F_REGION + F_STAGE_XI;
+                uint8_t* erow = slot + SLOT_E + i * 16;
+                uint8_t* xrow = slot + SLOT_XI + i * 16;
 #pragma unroll 1
                 for (int c0 = 0; c0 < DK + DV; c0 += 32) {
                     uint32_t rr[32];
                     tmem_ld32(RA + lane_base + c0, rr);
                     tmem_ld_wait();
-                    uint8_t* dst = (c0 < DK) ? sE : sXi;
-                    const int col8 = ((c0 < DK) ? c0 : c0 - DK) >> 3;
+                    uint8_t* dst = (c0 < DK) ? erow + (c0 >> 3) * 2048 : xrow + ((c0 - DK) >> 3) * 2048;
 #pragma unroll
-                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + chunk_off(i, col8 + j8, 128)) = pack8(rr + 8 * j8, 1.f);
+                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + j8 * 2048) = pack8(rr + 8 * j8, 1.f);
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
-            fence_async_smem();
-            mbar_arrive(&bar[B_STAGED]);
-            PF_LAP(22);
+            PF_LAP(2);
             // ---- Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t]: row i of the Qt image, straight into the ring
             {
-                uint8_t* qrow = slot + SLOT_QT + i * 128;
+                uint8_t* qrow = slot + SLOT_QT + i * 16;
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t rr[32];
@@ -563,10 +574,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                             const float2 qf = __half22float2(*reinterpret_cast<const __half2*>(&qq));
                             w4[j] = pack_h2(__uint_as_float(rr[8 * j8 + 2 * j]) + qf.x, __uint_as_float(rr[8 * j8 + 2 * j + 1]) + qf.y);
                         }
-                        *(uint4*)(qrow + (((((c0 >> 3) + j8)) ^ (i & 7)) << 4)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                        *(uint4*)(qrow + ((c0 >> 3) + j8) * 2048) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
                 }
             }
+            PF_LAP(3);
             // ---- OI^T[j][t] -> OI[t][j] (fp32), straight into the ring
             {
                 float* oi = (float*)(slot + SLOT_OI) + i;
@@ -584,8 +596,9 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_before();
             mbar_arrive(&bar[B_D4FREE]);
             mbar_arrive(&bar[B_OUTDONE]);
-            PF_LAP(23);
+            PF_LAP(4);
         }
+        PF_LAP_FLUSH(2);
     } else if (warp == 12) {
         // ------------------------------------------------ TMA loads -------------------------------------------
         if (lane == 0) {
@@ -594,9 +607,8 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 const int b = j & 1;
                 int seq, c;
                 item(j, seq, c);
-                // K: its region was last read by MMA3 of chunk j-2 (n = 64: and held part of that chunk's Xi image)
+                // K and V: their regions were last read by the MMAs of chunk j-2
                 if (j >= 2 && !PF_WAIT(B_D34DONE, (j - 2) & 1, 131)) return;
-                if (N == 64 && j >= 2 && !PF_WAIT(B_VFREE + b, ((j >> 1) - 1) & 1, 134)) return;
                 mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
                 for (int h = 0; h < 2; ++h)
                     tma_load_3d(smem + b * F_REGION + K_OFF + h * KV_SLAB, &maps.k, 64 * h, c * C * r, seq, &bar[B_KFULL + b]);
@@ -604,9 +616,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 if (j >= 1 && (!PF_WAIT(B_P0DONE, (j - 1) & 1, 132) || !PF_WAIT(B_QCOPIED, (j - 1) & 1, 136))) return;
                 mbar_expect_tx(&bar[B_QFULL], (uint32_t)C * 256);
                 for (int h = 0; h < 2; ++h) tma_load_3d(smem + F_Q + h * 8192, &maps.q, 64 * h, c * C, seq, &bar[B_QFULL]);
-                // V: its region holds the Xi image of chunk j-2 until the bulk store has read it
-                if (j >= 2 && !PF_WAIT(B_VFREE + b, ((j >> 1) - 1) & 1, 133)) return;
-                if (N == 64 && j >= 2 && !PF_WAIT(B_XFREE + b, ((j >> 1) - 1) & 1, 135)) return;
                 mbar_expect_tx(&bar[B_VFULL + b], K_BYTES);
                 for (int h = 0; h < 2; ++h)
                     tma_load_3d(smem + b * F_REGION + V_OFF + h * KV_SLAB, &maps.v, 64 * h, c * C * r, seq, &bar[B_VFULL + b]);
@@ -633,15 +642,16 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     return;
                 if (k >= 1 && !PF_WAIT(B_RAFREE, (k - 1) & 1, 144)) return;
                 tc_fence_after();
+                PF_LAP(0);
                 gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
                 commit_uni(&bar[B_D2DONE]);
-                PF_LAP(30);
+                PF_LAP(1);
                 // P0^T = K Q^T   (RC was drained before MMA4 of chunk k-1 was issued)
                 if (!PF_WAIT(B_Q16, k & 1, 148)) return;
                 tc_fence_after();
+                PF_LAP(2);
                 gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
                 commit_uni(&bar[B_P0DONE]);
-                PF_LAP(32);
                 // G of the next chunk, from its bf16 tile
                 if (k + 1 < nk) {
                     if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
@@ -651,55 +661,50 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     gemm_uni<false, false, N, DK, N, N, true>(RB, k1_b, k1_b);
                     commit_uni(&bar[B_GDONE]);
                 }
-                PF_LAP(31);
+                PF_LAP(3);
                 // [E | Xi] = K^T [-W | Uh]
                 if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
                 tc_fence_after();
+                PF_LAP(4);
                 gemm_uni<true, true, DK + DV, N, N, N>(RA, k_b, x_b);
-                PF_LAP(33);
                 // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T   (RB: G of chunk k+1 must have been drained)
                 if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
+                PF_LAP(5);
                 if (k + 1 < nk && !PF_WAIT(B_GFREE, (k + 1) & 1, 151)) return;
                 tc_fence_after();
+                PF_LAP(6);
                 gemm_uni<true, true, 64, N, N, N>(RB, x_b, pt_b);
                 gemm_uni<true, true, 64, N, N, N>(RB + 64, v_b, pt_b);
                 commit_uni(&bar[B_D34DONE]);
-                PF_LAP(34);
+                PF_LAP(7);
             }
+            PF_LAP_FLUSH(4);
         }
     } else {
-        // ------------------------------------------------ store warp: staging -> ring, flags -----------------
+        // ------------------------------------------------ flag warp: ring back-pressure, ready flags ---------
         if (lane == 0) {
 #pragma unroll 1
             for (int k = 0; k < nk; ++k) {
-                const int b = k & 1;
                 int seq, c;
                 item(k, seq, c);
                 const int slot_i = c % g.R;
-                uint8_t* slot = ws.ring + ((size_t)seq * g.R + slot_i) * SLOT_BYTES;
                 // the scan must be done with the chunk that used this slot before
                 if (c >= g.R && !flag_wait_ge(&ws.consumed[seq], c - g.R + 1, err, 161)) return;
                 mbar_arrive(&bar[B_SLOTOK]);
-                PF_LAP(60);
-                if (!PF_WAIT(B_STAGED, k & 1, 162)) return;
-                PF_LAP(61);
-                bulk_store(slot + SLOT_E, smem + b * F_REGION, DK * DK * 2);
-                bulk_store(slot + SLOT_XI, smem + b * F_REGION + F_STAGE_XI, DK * DV * 2);
-                bulk_commit();
-                bulk_wait_read_all();
-                mbar_arrive(&bar[B_XFREE + b]);
-                mbar_arrive(&bar[B_VFREE + b]);
-                PF_LAP(62);
-                bulk_wait_all();
+                PF_LAP(0);
                 if (!PF_WAIT(B_OUTDONE, k & 1, 163)) return;
-                fence_async_global();
+                PF_LAP(1);
                 __threadfence();
                 st_release_gpu(&ws.ready[seq * g.R + slot_i], c + 1);
-                PF_LAP(63);
+                PF_LAP(2);
             }
+            PF_LAP_FLUSH(5);
         }
     }
-    if (tim) atomicAdd(tim + 240 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));   // whole role, per warp
+    if (tim) {      // whole role, per warp: cycles and nanoseconds
+        atomicAdd(tim + 240 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));
+        atomicAdd(tim + 280 + (threadIdx.x >> 5), (unsigned long long)(globaltimer_ns() - t_ns));
+    }
 }
 
 // =============================================================================================================
@@ -712,8 +717,10 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     int* err = ws.status;
     unsigned long long* const tim = timing_slot(ws, seq == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416));
     const long long t_role = clock64();
+    const unsigned long long t_ns = tim ? globaltimer_ns() : 0ull;
     long long t_lap = t_role;
-    (void)t_lap;
+    long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    (void)t_lap; (void)lapacc;
     const uint32_t t_delta = tb, t_o = tb + 128;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
@@ -735,40 +742,43 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             // fp16 copy of the state: B operand of Delta, A operand of O^T
             bool ok = true;
             if (c >= 2) ok = PF_WAIT(B_S16FREE + buf, ((c >> 1) - 1) & 1, 201);
-            PF_LAP(40);
+            PF_LAP(0);
             uint8_t* sb = smem + S_S16 + buf * 32768 + w * 16384 + i * 128;
 #pragma unroll
             for (int p = 0; p < 8; ++p)
                 *(uint4*)(sb + ((p ^ (i & 7)) << 4)) =
                     make_uint4(pack_h2(S[8 * p], S[8 * p + 1]), pack_h2(S[8 * p + 2], S[8 * p + 3]),
                                pack_h2(S[8 * p + 4], S[8 * p + 5]), pack_h2(S[8 * p + 6], S[8 * p + 7]));
+            PF_LAP(1);
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_SREADY + buf]);
-            if (!named_bar_and(1 + w, 128, ok)) return;
-            PF_LAP(41);
-            // this half's Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j], issued by the half's first warp
-            if ((warp & 3) == 0) {
+            if (!named_bar_and(1, 256, ok)) return;
+            PF_LAP(2);
+            // Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j] for both halves, issued by warp 0
+            if (warp == 0) {
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                gemm_uni<false, true, 64, DK, 128, 128>(t_delta + 64 * w, smem_u32(smem + S_E + buf * 32768),
-                                                        smem_u32(smem + S_S16 + buf * 32768 + w * 16384));
-                commit_uni(&bar[B_DDONE + w]);
+                gemm_lay<L_NSK, L_SWMN, DV, DK, 128, 128>(t_delta, smem_u32(smem + S_E + buf * 32768),
+                                                          smem_u32(smem + S_S16 + buf * 32768));
+                commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
             }
+            PF_LAP(3);
             if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
-            if (!PF_WAIT(B_DDONE + w, c & 1, 202)) return;
+            PF_LAP(4);
+            if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
-            PF_LAP(42);
-            // S^T += Delta^T + Xi   (row i, columns 64w..64w+63; Xi from its swizzled image)
-            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + i * 128;
+            PF_LAP(5);
+            // S^T += Delta^T + Xi   (row i, columns 64w..64w+63; Xi from its column-group image)
+            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + i * 16;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(t_delta + lane_base + 64 * w + c0, rr);
                 uint4 xi[4];
 #pragma unroll
-                for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((((c0 >> 3) + p) ^ (i & 7)) << 4));
+                for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((c0 >> 3) + p) * 2048);
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
@@ -781,8 +791,9 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
-            PF_LAP(43);
+            PF_LAP(6);
         }
+        PF_LAP_FLUSH(8 + w);
         if (S_final)
 #pragma unroll
             for (int j = 0; j < 64; j += 4) *(float4*)(S_final + srow + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
@@ -810,7 +821,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             float* orow = O + ((long long)seq * g.L + (long long)c * g.C) * DV + j;
             if (!PF_WAIT(B_ODONE + ob, (c >> 1) & 1, 212)) return;
             tc_fence_after();
-            PF_LAP(45);
+            PF_LAP(0);
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
@@ -822,10 +833,11 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             }
             tc_fence_before();
             mbar_arrive(&bar[B_OFREE + ob]);
-            PF_LAP(46);
+            PF_LAP(1);
             if (c + 1 < NC && !fetch_oi(c + 1)) return;
-            PF_LAP(47);
+            PF_LAP(2);
         }
+        PF_LAP_FLUSH(10);
     } else if (warp == 12) {
         // ------------------------------------------------ producer: ring -> shared memory ----------------------
         if (lane == 0) {
@@ -847,38 +859,43 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 if (c >= 2 && !PF_WAIT(B_XIEMPTY + b, ((c >> 1) - 1) & 1, 224)) return;
                 mbar_expect_tx(&bar[B_XIFULL + b], DK * DV * 2);
                 bulk_load(smem + S_XI + b * 32768, slot + SLOT_XI, DK * DV * 2, &bar[B_XIFULL + b]);
+                PF_LAP(0);
                 if (c >= 2 && !PF_WAIT(B_QTEMPTY + b, ((c >> 1) - 1) & 1, 223)) return;
                 mbar_expect_tx(&bar[B_QTFULL + b], DK * 128);
                 bulk_load(smem + S_QT + b * 16384, slot + SLOT_QT, DK * 128, &bar[B_QTFULL + b]);
-                PF_LAP(50);
+                PF_LAP(1);
                 if (c + 1 < NC && !load_e(c + 1)) return;
-                PF_LAP(51);
+                PF_LAP(2);
             }
+            PF_LAP_FLUSH(11);
         }
     } else if (warp == 13) {
         // ------------------------------------------------ O^T MMA issue (whole warp), consumed reports --------
 #pragma unroll 1
         for (int c = 0; c < NC; ++c) {
             const int buf = c & 1, ob = c & 1;
-            PF_LAP(70);
             if (!PF_WAIT(B_SREADY + buf, (c >> 1) & 1, 232) || !PF_WAIT(B_QTFULL + ob, (c >> 1) & 1, 234)) return;
             if (c >= 2 && !PF_WAIT(B_OFREE + ob, ((c >> 1) - 1) & 1, 233)) return;
             tc_fence_after();
-            PF_LAP(71);
+            PF_LAP(0);
             // O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
-            gemm_uni<true, true, 64, DK, 128, 128>(t_o + ob * 64, smem_u32(smem + S_S16 + buf * 32768), smem_u32(smem + S_QT + ob * 16384));
+            gemm_lay<L_SWMN, L_NSMN, 64, DK, 128, 128>(t_o + ob * 64, smem_u32(smem + S_S16 + buf * 32768), smem_u32(smem + S_QT + ob * 16384));
             commit_uni(&bar[B_ODONE + ob]);
             commit_uni(&bar[B_QTEMPTY + ob]);
             commit_uni(&bar[B_S16FREE + buf]);
-            PF_LAP(72);
+            PF_LAP(1);
             // the output warps are done with chunk c-2, hence the chain with chunk c-3: chunks < c-2 are
             // consumed and their ring slots may be rewritten
             if (c >= 2 && lane == 0) st_release_gpu(&ws.consumed[seq], c - 2);
             __syncwarp();
-            PF_LAP(73);
+            PF_LAP(2);
         }
+        PF_LAP_FLUSH(12);
     }
-    if (tim) atomicAdd(tim + 260 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));   // whole role, per warp
+    if (tim) {
+        atomicAdd(tim + 260 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));
+        atomicAdd(tim + 300 + (threadIdx.x >> 5), (unsigned long long)(globaltimer_ns() - t_ns));
+    }
 }
 
 template <int N>
@@ -898,7 +915,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     if (tid == 0) {
         if (is_scan) {
             for (int x = 0; x < 2; ++x) {
-                mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 2);
+                mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
                 mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
                 mbar_init(&bar[B_SREADY + x], 256); mbar_init(&bar[B_S16FREE + x], 1);
@@ -909,14 +926,13 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
                 mbar_init(&bar[B_KFULL + x], 1); mbar_init(&bar[B_VFULL + x], 1);
                 mbar_init(&bar[B_K16 + x], 128); mbar_init(&bar[B_V16 + x], 128);
                 mbar_init(&bar[B_XREADY + x], 128);
-                mbar_init(&bar[B_XFREE + x], 1); mbar_init(&bar[B_VFREE + x], 1);
             }
             mbar_init(&bar[B_QFULL], 1); mbar_init(&bar[B_Q16], 128);
             mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128);
             mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 128);
             mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 128);
             mbar_init(&bar[B_D34DONE], 1); mbar_init(&bar[B_D4FREE], 128); mbar_init(&bar[B_RAFREE], 128);
-            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_STAGED], 128); mbar_init(&bar[B_OUTDONE], 128);
+            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_OUTDONE], 128);
             mbar_init(&bar[B_SLOTOK], 1);
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);

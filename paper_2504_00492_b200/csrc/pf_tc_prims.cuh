@@ -83,15 +83,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t p
     atomicCAS(err_flag, 0, code);
     return false;
 }
-// `tim` (diagnostic builds only, else null): per-code accumulators of the cycles spent waiting.
-__device__ __forceinline__ bool mbar_wait_clk(uint64_t* bar, uint32_t parity, int* err_flag, int code,
-                                              unsigned long long* tim = nullptr) {
-    if (tim) {      // (one try_wait may itself block for a while before it reports)
-        const long long t0 = clock64();
-        const bool ok = mbar_try_wait(bar, parity) || mbar_wait_slow(smem_u32(bar), parity, err_flag, code);
-        atomicAdd(tim + code, (unsigned long long)(clock64() - t0));
-        return ok;
-    }
+__device__ __forceinline__ bool mbar_wait_clk(uint64_t* bar, uint32_t parity, int* err_flag, int code) {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(smem_u32(bar), parity, err_flag, code);
 }
@@ -295,18 +287,33 @@ __device__ __forceinline__ bool elect_one() {
     asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
     return pred != 0;
 }
-template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
-__device__ __forceinline__ void gemm_uni(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
+// Operand layouts: 128-byte swizzled slabs (SW) or unswizzled column groups (NS), K-major or MN-major.
+enum { L_SWK = 0, L_SWMN = 1, L_NSK = 2, L_NSMN = 3 };
+template <int LAY, int ROWS>
+__device__ __forceinline__ uint64_t desc_of(uint32_t base) {
+    return LAY == L_SWK ? desc_kmajor(base) : LAY == L_SWMN ? desc_mnmajor(base, (uint32_t)ROWS * 128u)
+         : LAY == L_NSK ? desc_ns_kmajor(base, ROWS) : desc_ns_mnmajor(base, ROWS);
+}
+template <int LAY, int ROWS>
+__device__ __forceinline__ constexpr uint32_t kstep_off(int kk) {
+    return LAY == L_SWK ? (uint32_t)(kk >> 2) * (uint32_t)ROWS * 128u + (uint32_t)(kk & 3) * 32u
+         : LAY == L_SWMN ? (uint32_t)kk * 2048u
+         : LAY == L_NSK ? (uint32_t)kk * 2u * (uint32_t)ROWS * 16u : (uint32_t)kk * 256u;
+}
+template <int AL, int BL, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
+__device__ __forceinline__ void gemm_lay(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
+    constexpr bool A_MN = (AL == L_SWMN || AL == L_NSMN), B_MN = (BL == L_SWMN || BL == L_NSMN);
     constexpr uint32_t idesc = make_idesc(NCOLS, A_MN, B_MN, false) | (BF16 ? ((1u << 7) | (1u << 10)) : 0u);
-    const uint64_t a0 = A_MN ? desc_mnmajor(a_base, (uint32_t)A_ROWS * 128u) : desc_kmajor(a_base);
-    const uint64_t b0 = B_MN ? desc_mnmajor(b_base, (uint32_t)B_ROWS * 128u) : desc_kmajor(b_base);
+    const uint64_t a0 = desc_of<AL, A_ROWS>(a_base), b0 = desc_of<BL, B_ROWS>(b_base);
 #pragma unroll
     for (int kk = 0; kk < KDIM / 16; ++kk) {
-        const uint32_t a_off = A_MN ? (uint32_t)kk * 2048u : (uint32_t)(kk >> 2) * (uint32_t)A_ROWS * 128u + (uint32_t)(kk & 3) * 32u;
-        const uint32_t b_off = B_MN ? (uint32_t)kk * 2048u : (uint32_t)(kk >> 2) * (uint32_t)B_ROWS * 128u + (uint32_t)(kk & 3) * 32u;
-        const uint64_t ad = a0 + (uint64_t)(a_off >> 4), bd = b0 + (uint64_t)(b_off >> 4);
+        const uint64_t ad = a0 + (uint64_t)(kstep_off<AL, A_ROWS>(kk) >> 4), bd = b0 + (uint64_t)(kstep_off<BL, B_ROWS>(kk) >> 4);
         if (elect_one()) mma_f16(d_tmem, ad, bd, idesc, kk > 0);
     }
+}
+template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
+__device__ __forceinline__ void gemm_uni(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
+    gemm_lay<A_MN ? L_SWMN : L_SWK, B_MN ? L_SWMN : L_SWK, NCOLS, KDIM, A_ROWS, B_ROWS, BF16>(d_tmem, a_base, b_base);
 }
 __device__ __forceinline__ void commit_uni(uint64_t* bar) {
     if (elect_one()) mma_commit(bar);
