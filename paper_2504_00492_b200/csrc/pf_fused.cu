@@ -34,8 +34,8 @@
 // shared memory in a form the MMA descriptors read directly.
 //
 // A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns; warp 0
-// issues the Delta MMA for both halves), warps 8-11 add OI and write O, warp 12 streams
-// the E / Xi / Qt images in with bulk copies, warp 13 issues the O^T MMAs and reports consumed chunks.
+// issues the chunk's Delta and O^T MMAs), warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt
+// images in with bulk copies and is the only poller of the ready flags, warp 13 reports consumed chunks.
 //
 // Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
 // deliberately kept rolled: the instruction footprint of fifteen differently-specialised warps matters.
@@ -124,8 +124,8 @@ enum {
     B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
-    B_SREADY = 44,    // [2 buffers] chain: fp16 copy of the state published (256 arrivals)
-    B_S16FREE = 46,   // [2 buffers] mma: the O^T MMA that reads the copy is complete
+    B_ORPT = 44,      // [2] output warps: chunk finished (for the consumed report)
+    B_S16FREE = 46,   // [2 buffers] mma: the MMAs that read the fp16 copy of the state are complete
     B_DDONE = 48,     // Delta complete
     B_ODONE = 50,     // [2] mma: O^T complete
     B_OFREE = 52,     // [2] output warps: O^T drained
@@ -725,6 +725,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
     const int* ready = ws.ready + seq * g.R;
+    volatile int* vis = (volatile int*)(smem + F_BAR + B_COUNT * 8 + 8);   // chunks whose ready flag the producer has acquired
 
     if (warp < 8) {
         // ------------------------------------------------ chain: the state lives here -------------------------
@@ -752,17 +753,24 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             PF_LAP(1);
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(&bar[B_SREADY + buf]);
             if (!named_bar_and(1, 256, ok)) return;
             PF_LAP(2);
-            // Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j] for both halves, issued by warp 0
+            // warp 0 issues both products that read this copy of the state:
+            //   Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j]   and   O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
             if (warp == 0) {
+                const uint32_t s_b = smem_u32(smem + S_S16 + buf * 32768);
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                gemm_lay<L_NSK, L_SWMN, DV, DK, 128, 128>(t_delta, smem_u32(smem + S_E + buf * 32768),
-                                                          smem_u32(smem + S_S16 + buf * 32768));
+                gemm_lay<L_NSK, L_SWMN, DV, DK, 128, 128>(t_delta, smem_u32(smem + S_E + buf * 32768), s_b);
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
+                if (!PF_WAIT(B_QTFULL + buf, (c >> 1) & 1, 234)) return;
+                if (c >= 2 && !PF_WAIT(B_OFREE + buf, ((c >> 1) - 1) & 1, 233)) return;
+                tc_fence_after();
+                gemm_lay<L_SWMN, L_NSMN, 64, DK, 128, 128>(t_o + buf * 64, s_b, smem_u32(smem + S_QT + buf * 16384));
+                commit_uni(&bar[B_ODONE + buf]);
+                commit_uni(&bar[B_QTEMPTY + buf]);
+                commit_uni(&bar[B_S16FREE + buf]);
             }
             PF_LAP(3);
             if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
@@ -803,8 +811,9 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
         const int j = tid - 256;
         float a[64];
         auto fetch_oi = [&](int c) -> bool {
+            // (the producer warp has acquired the chunk's ready flag once *vis > c)
             int ok = 1;
-            if (lane == 0) ok = flag_wait_ge(&ready[c % g.R], c + 1, err, 211) ? 1 : 0;
+            if (lane == 0) ok = smem_wait_ge(vis, c + 1, err, 211) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) return false;
             const int Cv = min(g.C, g.L - c * g.C);
@@ -833,6 +842,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             }
             tc_fence_before();
             mbar_arrive(&bar[B_OFREE + ob]);
+            mbar_arrive(&bar[B_ORPT + ob]);
             PF_LAP(1);
             if (c + 1 < NC && !fetch_oi(c + 1)) return;
             PF_LAP(2);
@@ -845,6 +855,8 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 const int st = c & 1;
                 if (!flag_wait_ge(&ready[c % g.R], c + 1, err, 222)) return false;
                 fence_async_global();
+                __threadfence_block();
+                *vis = c + 1;
                 if (c >= 2 && !PF_WAIT(B_EEMPTY + st, ((c >> 1) - 1) & 1, 221)) return false;
                 mbar_expect_tx(&bar[B_EFULL + st], DK * DK * 2);
                 bulk_load(smem + S_E + st * 32768, ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_E, DK * DK * 2, &bar[B_EFULL + st]);
@@ -870,27 +882,19 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             PF_LAP_FLUSH(11);
         }
     } else if (warp == 13) {
-        // ------------------------------------------------ O^T MMA issue (whole warp), consumed reports --------
+        // ------------------------------------------------ consumed reports ------------------------------------
+        // Once the output warps are done with chunk c, chunks < c are consumed (the chain finished chunk c-1
+        // before it published the state for chunk c) and their ring slots may be rewritten.
+        if (lane == 0) {
 #pragma unroll 1
-        for (int c = 0; c < NC; ++c) {
-            const int buf = c & 1, ob = c & 1;
-            if (!PF_WAIT(B_SREADY + buf, (c >> 1) & 1, 232) || !PF_WAIT(B_QTFULL + ob, (c >> 1) & 1, 234)) return;
-            if (c >= 2 && !PF_WAIT(B_OFREE + ob, ((c >> 1) - 1) & 1, 233)) return;
-            tc_fence_after();
-            PF_LAP(0);
-            // O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
-            gemm_lay<L_SWMN, L_NSMN, 64, DK, 128, 128>(t_o + ob * 64, smem_u32(smem + S_S16 + buf * 32768), smem_u32(smem + S_QT + ob * 16384));
-            commit_uni(&bar[B_ODONE + ob]);
-            commit_uni(&bar[B_QTEMPTY + ob]);
-            commit_uni(&bar[B_S16FREE + buf]);
-            PF_LAP(1);
-            // the output warps are done with chunk c-2, hence the chain with chunk c-3: chunks < c-2 are
-            // consumed and their ring slots may be rewritten
-            if (c >= 2 && lane == 0) st_release_gpu(&ws.consumed[seq], c - 2);
-            __syncwarp();
-            PF_LAP(2);
+            for (int c = 0; c < NC; ++c) {
+                if (!PF_WAIT(B_ORPT + (c & 1), (c >> 1) & 1, 232)) return;
+                PF_LAP(0);
+                st_release_gpu(&ws.consumed[seq], c);
+                PF_LAP(1);
+            }
+            PF_LAP_FLUSH(12);
         }
-        PF_LAP_FLUSH(12);
     }
     if (tim) {
         atomicAdd(tim + 260 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));
@@ -918,7 +922,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
                 mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
                 mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
-                mbar_init(&bar[B_SREADY + x], 256); mbar_init(&bar[B_S16FREE + x], 1);
+                mbar_init(&bar[B_ORPT + x], 128); mbar_init(&bar[B_S16FREE + x], 1);
                 mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
             }
         } else {
@@ -938,6 +942,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.v);
         }
+        *(volatile int*)(smem + F_BAR + B_COUNT * 8 + 8) = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base_s, 512);

@@ -137,6 +137,22 @@ static __device__ __noinline__ bool flag_wait_ge(const int* p, int want, int* er
     return false;
 }
 
+// Waits until a shared-memory counter reaches `want` (written by another warp of the CTA after
+// __threadfence_block()), bounded by elapsed cycles.
+static __device__ __noinline__ bool smem_wait_ge(volatile int* p, int want, int* err_flag, int code) {
+    if (*p >= want) { __threadfence_block(); return true; }
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (*p >= want) { __threadfence_block(); return true; }
+        if ((it & 255u) == 0) {
+            if (clock64() - t0 > WAIT_CYCLES) break;
+            if ((it & 4095u) == 0 && *(volatile int*)err_flag != 0) return false;
+        }
+    }
+    atomicCAS(err_flag, 0, code);
+    return false;
+}
+
 // ---- proxies / fences ----------------------------------------------------------------------------
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
