@@ -167,7 +167,8 @@ int pf_profile_read(int idx, char* name, int name_cap, float* ms);
  *   D[128][N] (fp32) = (+-A) * B^T  over a contraction of 128, fp16 operands staged in shared memory.
  * variant bit 0: A is given as [k][m] (MN-major) instead of [m][k]; bit 1: B is given as [k][n]
  * instead of [n][k]; bit 2: negate A; bits 3 / 4: A / B staged unswizzled (column groups of 8) instead of
- * 128-byte swizzled.  A is 128x128 fp16, B is N x 128 (or 128 x N) fp16, N a multiple
+ * 128-byte swizzled; bit 5: A (given as [m][k]) is placed in tensor memory instead of shared memory.
+ * A is 128x128 fp16, B is N x 128 (or 128 x N) fp16, N a multiple
  * of 16 in [16, 256].  Device pointers.  Synchronises the stream and allocates; for tests only. */
 int pf_tc_selftest(int variant, const void* A, const void* B, float* D, int N, void* stream);
 

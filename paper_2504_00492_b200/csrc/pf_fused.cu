@@ -7,11 +7,11 @@
 //       (chunk 0 of every sequence, then chunk 1, ...) and build for each chunk, from Theorem 3.2,
 //           X  = (I + Mstrict (.) (K K^T diag(beta)))^{-1}          (so that T' = diag(beta) X)
 //           W  = diag(beta) X K,   Uh = diag(beta) X V
-//           E  = -K^T W,  Xi = K^T Uh                                (the chunk flow of Proposition 2.1)
+//           E  = -K^T W,  Xi^T = Uh^T K                              (the chunk flow of Proposition 2.1)
 //           Qt = Q - P W (stored transposed),  OI = P Uh,            P = (Q K^T) (.) Mincl
 //       and store (E, Qt, Xi, OI) into slot (chunk mod R) of the sequence's ring;
 //   scan CTAs (one per sequence) carry the state over the chunks,
-//           O^T = OI^T + S Qt^T,      S^T <- S^T + E S^T + Xi,
+//           O^T = OI^T + S Qt^T,      S <- S + S E^T + Xi^T,
 //       reading each slot as soon as its flag is set and freeing it for the flow CTAs afterwards.
 //
 // The ring (R slots of 112 KB per sequence) is rewritten in place, so the hand-off never has to reach HBM:
@@ -24,7 +24,7 @@
 //   warp 12             TMA loads (K and V double-buffered, Q single)
 //   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
 //   warp 14             ring back-pressure and ready flags
-// Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi]; RB = [256,384) holds G of the NEXT
+// Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi^T]; RB = [256,384) holds G of the NEXT
 // chunk and then [Qt^T | OI^T] of the current one; RC = [384,448) holds P0^T.
 // G is formed from the bf16 tiles as they land (both operands raw); every other product has a derived fp16
 // operand, so K, V and Q are converted to fp16 in place, off the critical path.
@@ -33,9 +33,11 @@
 // consecutive rows then writes 512 contiguous bytes per store, and the scan's bulk copies bring them into
 // shared memory in a form the MMA descriptors read directly.
 //
-// A scan CTA: warps 0-7 own the state (row i of S^T per thread, d_v split in two halves of 64 columns; warp 0
-// issues the chunk's Delta and O^T MMAs), warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt
-// images in with bulk copies and is the only poller of the ready flags, warp 13 reports consumed chunks.
+// A scan CTA: warps 0-7 own the state (row j of S per thread, d_k split in two halves of 64 columns).  Each
+// chunk they write an fp16 copy of it into TENSOR memory, where it is the A operand of both of the chunk's
+// products (Delta = S E^T and O^T = S Qt^T, issued by warp 0), so the serial step never goes through shared
+// memory.  Warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt images in with bulk copies and is
+// the only poller of the ready flags, warp 13 reports consumed chunks.
 //
 // Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
 // deliberately kept rolled: the instruction footprint of fifteen differently-specialised warps matters.
@@ -57,7 +59,7 @@ constexpr int DK = 128, DV = 128;
 // ---- ring slot layout (bytes) ---------------------------------------------------------------------------
 constexpr uint32_t SLOT_E = 0;                          // E image : fp16 [16 groups i'/8][128 rows i][16 B]  (K-major A)
 constexpr uint32_t SLOT_QT = SLOT_E + DK * DK * 2;      // Qt image: fp16 [ 8 groups t/8 ][128 rows i][16 B]  (MN-major B)
-constexpr uint32_t SLOT_XI = SLOT_QT + DK * 128;        // Xi image: fp16 [16 groups j/8 ][128 rows i][16 B]
+constexpr uint32_t SLOT_XI = SLOT_QT + DK * 128;        // Xi^T    : fp16 [16 groups i/8 ][128 rows j][16 B]
 constexpr uint32_t SLOT_OI = SLOT_XI + DK * DV * 2;     // OI      : fp32 [64 rows t][128 cols j]
 constexpr uint32_t SLOT_BYTES = SLOT_OI + 64 * DV * 4;  // 114688
 
@@ -91,8 +93,7 @@ constexpr int SMEM_BYTES = F_BAR + 512;         // 230912
 constexpr int S_E = 0;                          // 2 x 32 KB  E images
 constexpr int S_XI = S_E + 2 * 32768;           // 2 x 32 KB  Xi images
 constexpr int S_QT = S_XI + 2 * 32768;          // 2 x 16 KB  Qt images
-constexpr int S_S16 = S_QT + 2 * 16384;         // 2 x 32 KB  fp16 copies of the state
-static_assert(S_S16 + 2 * 32768 <= F_BAR, "scan role fits below the barrier block");
+static_assert(S_QT + 2 * 16384 <= F_BAR, "scan role fits below the barrier block");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // barriers (indices into the uint64_t block at F_BAR)
@@ -125,7 +126,7 @@ enum {
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
     B_ORPT = 44,      // [2] output warps: chunk finished (for the consumed report)
-    B_S16FREE = 46,   // [2 buffers] mma: the MMAs that read the fp16 copy of the state are complete
+    B_S16FREE = 46,   // [2 buffers] mma: the MMAs that read that fp16 copy of the state are complete
     B_DDONE = 48,     // Delta complete
     B_ODONE = 50,     // [2] mma: O^T complete
     B_OFREE = 52,     // [2] output warps: O^T drained
@@ -540,7 +541,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_after();
             if (!ok) return;
             PF_LAP(1);
-            // ---- [E | Xi] from RA: row i of both images, one 16-byte piece per column group
+            // ---- [E | Xi^T] from RA: row i of E and row j = i of Xi^T, one 16-byte piece per column group
             {
                 uint8_t* erow = slot + SLOT_E + i * 16;
                 uint8_t* xrow = slot + SLOT_XI + i * 16;
@@ -662,11 +663,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     commit_uni(&bar[B_GDONE]);
                 }
                 PF_LAP(3);
-                // [E | Xi] = K^T [-W | Uh]
+                // E = K^T (-W)  (lanes i, columns i'),   Xi^T = Uh^T K  (lanes j, columns i)
                 if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
                 tc_fence_after();
                 PF_LAP(4);
-                gemm_uni<true, true, DK + DV, N, N, N>(RA, k_b, x_b);
+                gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
+                gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
                 // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T   (RB: G of chunk k+1 must have been drained)
                 if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
                 PF_LAP(5);
@@ -721,7 +723,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     long long t_lap = t_role;
     long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     (void)t_lap; (void)lapacc;
-    const uint32_t t_delta = tb, t_o = tb + 128;
+    const uint32_t t_delta = tb, t_o = tb + 128, t_a = tb + 256;     // Delta | 2 x O^T | 2 x fp16 state
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
     const int* ready = ws.ready + seq * g.R;
@@ -729,45 +731,43 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
 
     if (warp < 8) {
         // ------------------------------------------------ chain: the state lives here -------------------------
-        const int w = warp >> 2, i = tid & 127;
+        // thread (w, j): row j of S, columns i = 64w .. 64w+63
+        const int w = warp >> 2, j = tid & 127;
         float S[64];
-        const long long srow = ((long long)seq * DK + i) * DV + 64 * w;
+        const long long sbase = ((long long)seq * DK + 64 * w) * DV + j;
 #pragma unroll
-        for (int j = 0; j < 64; j += 4) {
-            float4 v4 = S0 ? *(const float4*)(S0 + srow + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-            S[j] = v4.x; S[j + 1] = v4.y; S[j + 2] = v4.z; S[j + 3] = v4.w;
-        }
+        for (int ii = 0; ii < 64; ++ii) S[ii] = S0 ? S0[sbase + (long long)ii * DV] : 0.f;
 #pragma unroll 1
         for (int c = 0; c < NC; ++c) {
             const int buf = c & 1;
-            // fp16 copy of the state: B operand of Delta, A operand of O^T
+            // fp16 copy of the state into tensor memory (A operand of Delta and of O^T): 32 packed columns per thread
             bool ok = true;
             if (c >= 2) ok = PF_WAIT(B_S16FREE + buf, ((c >> 1) - 1) & 1, 201);
+            tc_fence_after();
             PF_LAP(0);
-            uint8_t* sb = smem + S_S16 + buf * 32768 + w * 16384 + i * 128;
+            {
+                uint32_t pk[32];
 #pragma unroll
-            for (int p = 0; p < 8; ++p)
-                *(uint4*)(sb + ((p ^ (i & 7)) << 4)) =
-                    make_uint4(pack_h2(S[8 * p], S[8 * p + 1]), pack_h2(S[8 * p + 2], S[8 * p + 3]),
-                               pack_h2(S[8 * p + 4], S[8 * p + 5]), pack_h2(S[8 * p + 6], S[8 * p + 7]));
+                for (int q = 0; q < 32; ++q) pk[q] = pack_h2(S[2 * q], S[2 * q + 1]);
+                tmem_st32(t_a + buf * 64 + 32 * w + lane_base, pk);
+                tmem_st_wait();
+            }
             PF_LAP(1);
-            fence_async_smem();
             tc_fence_before();
             if (!named_bar_and(1, 256, ok)) return;
             PF_LAP(2);
             // warp 0 issues both products that read this copy of the state:
-            //   Delta^T[i][j] = sum_i' E[i][i'] S^T[i'][j]   and   O^T[j][t] = sum_i S^T[i][j] Qt^T[i][t]
+            //   Delta[j][i] = sum_i' S[j][i'] E[i][i']   and   O^T[j][t] = sum_i S[j][i] Qt^T[i][t]
             if (warp == 0) {
-                const uint32_t s_b = smem_u32(smem + S_S16 + buf * 32768);
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                gemm_lay<L_NSK, L_SWMN, DV, DK, 128, 128>(t_delta, smem_u32(smem + S_E + buf * 32768), s_b);
+                gemm_ta<L_NSK, DK, DK, 128>(t_delta, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
                 if (!PF_WAIT(B_QTFULL + buf, (c >> 1) & 1, 234)) return;
                 if (c >= 2 && !PF_WAIT(B_OFREE + buf, ((c >> 1) - 1) & 1, 233)) return;
                 tc_fence_after();
-                gemm_lay<L_SWMN, L_NSMN, 64, DK, 128, 128>(t_o + buf * 64, s_b, smem_u32(smem + S_QT + buf * 16384));
+                gemm_ta<L_NSMN, 64, DK, 128>(t_o + buf * 64, t_a + buf * 64, smem_u32(smem + S_QT + buf * 16384));
                 commit_uni(&bar[B_ODONE + buf]);
                 commit_uni(&bar[B_QTEMPTY + buf]);
                 commit_uni(&bar[B_S16FREE + buf]);
@@ -778,8 +778,8 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
             PF_LAP(5);
-            // S^T += Delta^T + Xi   (row i, columns 64w..64w+63; Xi from its column-group image)
-            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + i * 16;
+            // S += Delta + Xi^T   (row j, columns 64w..64w+63; Xi^T from its column-group image)
+            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + j * 16;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
@@ -789,11 +789,11 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((c0 >> 3) + p) * 2048);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; j += 2) {
-                    const uint32_t wd = ((const uint32_t*)&xi[j >> 3])[(j & 7) >> 1];
+                for (int e = 0; e < 32; e += 2) {
+                    const uint32_t wd = ((const uint32_t*)&xi[e >> 3])[(e & 7) >> 1];
                     const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&wd));
-                    S[c0 + j] += __uint_as_float(rr[j]) + xv.x;
-                    S[c0 + j + 1] += __uint_as_float(rr[j + 1]) + xv.y;
+                    S[c0 + e] += __uint_as_float(rr[e]) + xv.x;
+                    S[c0 + e + 1] += __uint_as_float(rr[e + 1]) + xv.y;
                 }
             }
             tc_fence_before();
@@ -804,7 +804,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
         PF_LAP_FLUSH(8 + w);
         if (S_final)
 #pragma unroll
-            for (int j = 0; j < 64; j += 4) *(float4*)(S_final + srow + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+            for (int ii = 0; ii < 64; ++ii) S_final[sbase + (long long)ii * DV] = S[ii];
     } else if (warp < 12) {
         // ------------------------------------------------ output: O^T = OI^T + S Qt^T --------------------------
         // OI of the next chunk is fetched (into registers) while this chunk's MMA is awaited.

@@ -270,6 +270,29 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
         : "memory");
 }
+// Same with the A operand in tensor memory: lane m holds row m, 32-bit column c holds elements k = 2c (low
+// half) and 2c+1 (high half); one K = 16 step reads 8 columns.  The instruction descriptor must say K-major A.
+__device__ __forceinline__ void mma_f16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    const uint32_t acc = accumulate ? 1u : 0u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns, registers -> tensor memory (one full warp)
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // Arrives on `bar` when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -325,6 +348,18 @@ __device__ __forceinline__ void gemm_lay(uint32_t d_tmem, uint32_t a_base, uint3
     for (int kk = 0; kk < KDIM / 16; ++kk) {
         const uint64_t ad = a0 + (uint64_t)(kstep_off<AL, A_ROWS>(kk) >> 4), bd = b0 + (uint64_t)(kstep_off<BL, B_ROWS>(kk) >> 4);
         if (elect_one()) mma_f16(d_tmem, ad, bd, idesc, kk > 0);
+    }
+}
+// D[128 x NCOLS] = A * B^T with A (fp16, K-major, KDIM/2 packed columns) in tensor memory; whole warp, converged.
+template <int BL, int NCOLS, int KDIM, int B_ROWS>
+__device__ __forceinline__ void gemm_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base) {
+    constexpr bool B_MN = (BL == L_SWMN || BL == L_NSMN);
+    constexpr uint32_t idesc = make_idesc(NCOLS, false, B_MN, false);
+    const uint64_t b0 = desc_of<BL, B_ROWS>(b_base);
+#pragma unroll
+    for (int kk = 0; kk < KDIM / 16; ++kk) {
+        const uint64_t bd = b0 + (uint64_t)(kstep_off<BL, B_ROWS>(kk) >> 4);
+        if (elect_one()) mma_f16_ta(d_tmem, a_tmem + 8u * (uint32_t)kk, bd, idesc, kk > 0);
     }
 }
 template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>

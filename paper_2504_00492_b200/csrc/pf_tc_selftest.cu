@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
     __shared__ uint32_t tmem_base;
     const bool a_mn = variant & 1, b_mn = variant & 2, neg = variant & 4;
     const bool a_ns = variant & 8, b_ns = variant & 16;      // operand stored unswizzled (column groups of 8)
+    const bool a_tm = variant & 32;                          // A (K-major) in tensor memory instead of shared memory
     const int tid = threadIdx.x, warp = tid >> 5;
 
     // A is given row-major as [128][128] in both cases: K-major -> A[m][k]; MN-major -> A[k][m].
@@ -43,17 +44,40 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
         mbar_fence_init();
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(&tmem_base, 256);
+    if (warp == 0) tmem_alloc(&tmem_base, 512);
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base;
 
+    if (a_tm) {
+        // row m of A as 64 packed words into tensor memory columns [256, 320)   (the accumulator uses [0, N))
+        for (int half = 0; half < 2; ++half) {
+            uint32_t w[32];
+            for (int c = 0; c < 32; ++c) {
+                const __half2 h2 = __halves2half2(A[tid * 128 + 64 * half + 2 * c], A[tid * 128 + 64 * half + 2 * c + 1]);
+                w[c] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            tmem_st32(tb + 256 + 32 * half + ((uint32_t)(warp * 32) << 16), w);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
     if (tid == 0) {
         const uint32_t a_base = smem_u32(sA), b_base = smem_u32(sB);
         const int b_rows = b_mn ? 128 : N;
-        if (a_ns || b_ns) {
+        if (a_tm) {
+            const uint32_t idesc = make_idesc(N, false, b_mn, neg);
+            for (int kk = 0; kk < 8; ++kk) {
+                uint64_t bd;
+                if (b_ns) bd = b_mn ? desc_ns_mnmajor(b_base + kk * ns_kstep_mnmajor(), b_rows) : desc_ns_kmajor(b_base + kk * ns_kstep_kmajor(b_rows), b_rows);
+                else bd = b_mn ? desc_mnmajor(b_base + kk * 2048u, (uint32_t)b_rows * 128u) : desc_kmajor(b_base + (kk >> 2) * (uint32_t)b_rows * 128u + (kk & 3) * 32u);
+                mma_f16_ta(tb, tb + 256 + 8 * kk, bd, idesc, kk > 0);
+            }
+        } else if (a_ns || b_ns) {
             const uint32_t idesc = make_idesc(N, a_mn, b_mn, neg);
             for (int kk = 0; kk < 8; ++kk) {
                 uint64_t ad, bd;
@@ -82,7 +106,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 256);
+    if (warp == 0) tmem_dealloc(tb, 512);
 }
 
 }  // namespace
@@ -91,7 +115,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(int variant, const __h
 extern "C" int pf_tc_selftest(int variant, const void* A, const void* B, float* D, int N, void* stream) {
     using namespace pf;
     if (!A || !B || !D) return PF_ERR_INVALID;
-    if (variant < 0 || variant > 31) return PF_ERR_INVALID;
+    if (variant < 0 || variant > 63 || ((variant & 32) && (variant & 9))) return PF_ERR_INVALID;
     if (N < 16 || N > 256 || (N % 16)) return PF_ERR_UNSUPPORTED;
     int dev = 0, major = 0;
     PF_CUDA_TRY(cudaGetDevice(&dev));

@@ -5,7 +5,7 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("variant", list(range(8)) + [8, 9, 16, 18, 24, 27, 10, 17])
+@pytest.mark.parametrize("variant", list(range(8)) + [8, 9, 16, 18, 24, 27, 10, 17, 32, 34, 36, 48, 50])
 @pytest.mark.parametrize("N", [32, 64, 128, 192, 256])
 def test_tcgen05_gemm_variants(variant, N):
     from paper_2504_00492_b200 import binding
