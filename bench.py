@@ -62,6 +62,27 @@ def flops_per_chunk(w, tri: bool) -> dict:
     }
 
 
+# DRAM bytes (read + write) of one launch of the single-launch kernel from an ncu capture, valid only for the
+# kernel sources it was taken on (their hash is stored with it): {workload: (sha256 of the sources, bytes)}.
+NCU_TRAFFIC = {}
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("pf_fused.cu", "pf_tc_prims.cuh"):
+        with open(os.path.join(ROOT, "paper_2504_00492_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(w):
+    ent = NCU_TRAFFIC.get(w.name)
+    if not ent or ent[0] != kernel_source_hash():
+        return None        # no capture, or the kernel has changed since the counters were taken
+    return ent[1]
+
+
 class ClockSampler:
     """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -306,15 +327,29 @@ def main():
     roofline = None
     if prof:
         top = max(prof, key=prof.get)
-        steps_of = kernel_steps.get(top, list(fl_tri))
-        fl = G * sum(fl_tri[s] for s in steps_of)
-        achieved = fl / (prof[top] * 1e-3) / 1e12
-        bound = "alu" if top.startswith("simt") else "tensor"
-        # fp32 FFMA peak: 148 SMs x 128 lanes x 2 FLOP x max SM clock
-        peak = 148 * 128 * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12 if bound == "alu" else peaks["bf16_tflops"]
-        roofline = {"bound": bound, "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": None, "ms_per_launch": prof[top], "peaks": peak_kind,
-                    "flops_per_launch": fl, "flop_count": "triangular-aware", "kernel_ms": prof}
+        if top == "fused":
+            # The single-launch path does everything: its algorithmic traffic is one read of q, k, v, beta and one
+            # write of O; at the measured peaks that HBM time exceeds the tensor time of the dense FLOPs, so HBM is
+            # the roofline that binds (the tensor figure is printed beside it).
+            nbytes = th * alg_bytes_per_token_head(w)
+            achieved = nbytes / (prof[top] * 1e-3) / 1e9
+            fl_d = G * sum(fl_dense[k] for k in fl_dense if k != "solve")
+            roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(w), "ms_per_launch": prof[top],
+                        "peaks": peak_kind, "bytes_per_launch": nbytes,
+                        "tensor": {"tflops_dense": fl_d / (prof[top] * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                                   "frac": fl_d / (prof[top] * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+                        "kernel_ms": prof}
+        else:
+            steps_of = kernel_steps.get(top, list(fl_tri))
+            fl = G * sum(fl_tri[s] for s in steps_of)
+            achieved = fl / (prof[top] * 1e-3) / 1e12
+            bound = "alu" if top.startswith("simt") else "tensor"
+            # fp32 FFMA peak: 148 SMs x 128 lanes x 2 FLOP x max SM clock
+            peak = 148 * 128 * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12 if bound == "alu" else peaks["bf16_tflops"]
+            roofline = {"bound": bound, "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                        "frac": achieved / peak, "traffic": None, "ms_per_launch": prof[top], "peaks": peak_kind,
+                        "flops_per_launch": fl, "flop_count": "triangular-aware", "kernel_ms": prof}
 
     if rank == 0:
         cpu = None

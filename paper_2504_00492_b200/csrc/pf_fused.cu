@@ -19,8 +19,8 @@
 //
 // A flow CTA is software-pipelined over two chunks (15 warps):
 //   warps 0-3  "solve"  epilogue of G = K K^T (mask, column scaling, fp16) and the triangular inverse
-//   warps 4-7  "mid"    epilogues of [Uh | W] and P^T; bf16 -> fp16 conversion of K, V, Q
-//   warps 8-11 "out"    epilogues of [E | Xi] and [Qt^T | OI^T], stored straight into the ring
+//   warps 4-7  "mid"    Uh half of [Uh | W], Xi^T half of [E | Xi^T] (into the ring), bf16 -> fp16 of V and K
+//   warps 8-11 "out"    W half, P^T, E half and [Qt^T | OI^T] (into the ring), bf16 -> fp16 of Q
 //   warp 12             TMA loads (K and V double-buffered, Q single)
 //   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
 //   warp 14             ring back-pressure and ready flags
@@ -112,7 +112,8 @@ enum {
     B_WUREADY = 15,   // mid: W, Uh in shared memory (RA drained)
     B_P0DONE = 16,    // mma: P0^T complete
     B_PTREADY = 17,   // mid: P^T in shared memory (RC drained)
-    B_D34DONE = 18,   // mma: [E | Xi] and [Qt^T | OI^T] complete
+    B_D4DONE = 18,    // mma: [Qt^T | OI^T] complete (and everything issued before it)
+    B_RADONE = 29,    // mma: [E | Xi^T] complete
     B_D4FREE = 19,    // out: RB drained
     B_RAFREE = 20,    // out: RA drained
     B_QCOPIED = 25,   // out: Q copied into registers
@@ -125,7 +126,6 @@ enum {
     B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
-    B_ORPT = 44,      // [2] output warps: chunk finished (for the consumed report)
     B_S16FREE = 46,   // [2 buffers] mma: the MMAs that read that fp16 copy of the state are complete
     B_DDONE = 48,     // Delta complete
     B_ODONE = 50,     // [2] mma: O^T complete
@@ -328,7 +328,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
             bool ok = true;
-            if (k >= 2) ok = PF_WAIT(B_D34DONE, (k - 2) & 1, 101);     // W of chunk k-2 (in this X region) has been read
+            if (k >= 2) ok = PF_WAIT(B_D4DONE, (k - 2) & 1, 101);     // W of chunk k-2 (in this X region) has been read
             sB[m] = bm;     // (the beta half of chunk k-2 was last read by that chunk's [Uh | W] epilogue)
             ok = ok && PF_WAIT(B_GDONE, k & 1, 102);
             tc_fence_after();
@@ -409,51 +409,133 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
         }
         PF_LAP_FLUSH(0);
     } else if (warp < 8) {
-        // ------------------------------------------------ mid: [Uh | W] and P^T epilogues, conversions --------
+        // ------------------------------------------------ mid: Uh and Xi^T halves, conversions of V and K -----
         const int m = tid - 128;
-        const int tokm = m / r;
         const float* sBeta = (const float*)(smem + F_BETA);
-        uint8_t* sPT = smem + F_PT;
         if (nk > 0) {
-            // chunk 0: K after its Gram product has read the bf16 tile, V and Q as they land
-            if (!PF_WAIT(B_KFULL + 0, 0, 111) || !PF_WAIT(B_GDONE, 0, 110)) return;
-            cvt_region(smem + K_OFF, K_BYTES, m);
-            fence_async_smem();
-            mbar_arrive(&bar[B_K16 + 0]);
             if (!PF_WAIT(B_VFULL + 0, 0, 112)) return;
             cvt_region(smem + V_OFF, K_BYTES, m);
             fence_async_smem();
             mbar_arrive(&bar[B_V16 + 0]);
-            if (!PF_WAIT(B_QFULL, 0, 109)) return;
-            cvt_region(smem + F_Q, 16384, m);
+            // (K only once its Gram product has read the bf16 tile)
+            if (!PF_WAIT(B_KFULL + 0, 0, 111) || !PF_WAIT(B_GDONE, 0, 110)) return;
+            cvt_region(smem + K_OFF, K_BYTES, m);
             fence_async_smem();
-            mbar_arrive(&bar[B_Q16]);
+            mbar_arrive(&bar[B_K16 + 0]);
         }
 #pragma unroll 1
         for (int k = 0; k < nk; ++k) {
             const int b = k & 1, b1 = b ^ 1;
             int seq, c;
             item(k, seq, c);
-            const int Cv = min(C, g.L - c * C), nv = Cv * r;
-            // ---- RA = X [V | K]:  Uh = diag(beta) (X V) over V,  -W = -diag(beta) (X K) over X, fp16 operands
+            uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
+            // ---- RA = X [V | K], first half:  Uh = diag(beta) (X V), fp16, over V
             if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
             tc_fence_after();
             PF_LAP(0);
             {
                 const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
                 uint8_t* sU = smem + b * F_REGION + V_OFF;
-                uint8_t* sW = smem + b * F_REGION + X_OFF;
 #pragma unroll 1
-                for (int c0 = 0; c0 < DV + DK; c0 += 32) {
+                for (int c0 = 0; c0 < DV; c0 += 32) {
                     uint32_t rr[32];
                     tmem_ld32(RA + lane_base + c0, rr);
                     tmem_ld_wait();
                     if (m < N) {
-                        uint8_t* dst = (c0 < DV) ? sU : sW;
-                        const int col8 = ((c0 < DV) ? c0 : c0 - DV) >> 3;
-                        const float sc = (c0 < DV) ? bm : -bm;
 #pragma unroll
-                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + chunk_off(m, col8 + j8, N)) = pack8(rr + 8 * j8, sc);
+                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(sU + chunk_off(m, (c0 >> 3) + j8, N)) = pack8(rr + 8 * j8, bm);
+                    }
+                }
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(&bar[B_WUREADY]);
+            PF_LAP(1);
+            // ---- conversions for chunk k+1
+            if (k + 1 < nk) {
+                if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
+                PF_LAP(2);
+                cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
+                fence_async_smem();
+                mbar_arrive(&bar[B_V16 + b1]);
+                PF_LAP(3);
+                if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
+                PF_LAP(4);
+                cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
+                fence_async_smem();
+                mbar_arrive(&bar[B_K16 + b1]);
+                PF_LAP(5);
+            }
+            // ---- RA = [E | Xi^T], second half: row j = m of Xi^T, one 16-byte piece per column group, into the ring
+            if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
+            tc_fence_after();
+            PF_LAP(6);
+            {
+                uint8_t* xrow = slot + SLOT_XI + m * 16;
+#pragma unroll 1
+                for (int c0 = 0; c0 < DK; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RA + lane_base + DK + c0, rr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(xrow + ((c0 >> 3) + j8) * 2048) = pack8(rr + 8 * j8, 1.f);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&bar[B_RAFREE]);
+            mbar_arrive(&bar[B_OUTDONE]);
+            PF_LAP(7);
+        }
+        PF_LAP_FLUSH(1);
+    } else if (warp < 12) {
+        // ------------------------------------------------ out: W half, P^T, E / Qt / OI into the ring, Q ---------
+        const int i = tid - 256;
+        const int tokm = i / r;
+        const float* sBeta = (const float*)(smem + F_BETA);
+        uint8_t* sPT = smem + F_PT;
+        const uint8_t* sQ = smem + F_Q;
+        uint32_t qreg[32];      // column i of Q (fp16 pairs over t): lets the Q buffer take the next chunk early
+        auto q_prepare = [&](int k) -> bool {
+            // (a failed wait must not strand the others at the barrier: the barrier carries the outcome)
+            bool okq = PF_WAIT(B_QFULL, k & 1, 114);
+            if (okq) cvt_region(smem + F_Q, 16384, i);
+            fence_async_smem();
+            if (okq) mbar_arrive(&bar[B_Q16]);
+            if (!named_bar_and(3, 128, okq)) return false;
+            const uint8_t* qcol = sQ + (i >> 6) * 8192 + (i & 7) * 2;
+            const int ci = (i & 63) >> 3;
+#pragma unroll
+            for (int t = 0; t < 64; t += 2) {
+                const uint32_t lo = *(const uint16_t*)(qcol + t * 128 + ((ci ^ (t & 7)) << 4));
+                const uint32_t hi = *(const uint16_t*)(qcol + (t + 1) * 128 + ((ci ^ ((t + 1) & 7)) << 4));
+                qreg[t >> 1] = lo | (hi << 16);
+            }
+            mbar_arrive(&bar[B_QCOPIED]);
+            return true;
+        };
+        if (nk > 0 && !q_prepare(0)) return;
+#pragma unroll 1
+        for (int k = 0; k < nk; ++k) {
+            const int b = k & 1;
+            int seq, c;
+            item(k, seq, c);
+            const int Cv = min(C, g.L - c * C), nv = Cv * r;
+            uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
+            // ---- RA = X [V | K], second half:  -W = -diag(beta) (X K), fp16, over X
+            if (!PF_WAIT(B_D2DONE, k & 1, 125)) return;
+            tc_fence_after();
+            PF_LAP(0);
+            {
+                const float bm = (i < N) ? -sBeta[b * 128 + i] : 0.f;
+                uint8_t* sW = smem + b * F_REGION + X_OFF;
+#pragma unroll 1
+                for (int c0 = 0; c0 < DK; c0 += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(RA + lane_base + DV + c0, rr);
+                    tmem_ld_wait();
+                    if (i < N) {
+#pragma unroll
+                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(sW + chunk_off(i, (c0 >> 3) + j8, N)) = pack8(rr + 8 * j8, bm);
                     }
                 }
             }
@@ -462,25 +544,24 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             mbar_arrive(&bar[B_WUREADY]);
             PF_LAP(1);
             // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
-            if (k >= 1 && !PF_WAIT(B_D34DONE, (k - 1) & 1, 116)) return;
+            if (k >= 1 && !PF_WAIT(B_D4DONE, (k - 1) & 1, 116)) return;
             if (!PF_WAIT(B_P0DONE, k & 1, 117)) return;
             tc_fence_after();
-            PF_LAP(2);
 #pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(RC + lane_base + c0, rr);
                 tmem_ld_wait();
-                if (m < N) {
+                if (i < N) {
 #pragma unroll
                     for (int j8 = 0; j8 < 32; j8 += 8) {
                         float a[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const int t = c0 + j8 + j;
-                            a[j] = (tokm <= t && t < Cv && m < nv) ? __uint_as_float(rr[j8 + j]) : 0.f;
+                            a[j] = (tokm <= t && t < Cv && i < nv) ? __uint_as_float(rr[j8 + j]) : 0.f;
                         }
-                        *(uint4*)(sPT + chunk_off(m, (c0 + j8) >> 3, N)) =
+                        *(uint4*)(sPT + chunk_off(i, (c0 + j8) >> 3, N)) =
                             make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                     }
                 }
@@ -488,77 +569,29 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_PTREADY]);
-            PF_LAP(3);
-            // ---- conversions for chunk k+1 (K only once its Gram product has read the bf16 tile)
-            if (k + 1 < nk) {
-                if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
-                PF_LAP(4);
-                cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_K16 + b1]);
-                PF_LAP(5);
-                if (!PF_WAIT(B_QFULL, (k + 1) & 1, 114)) return;
-                cvt_region(smem + F_Q, 16384, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_Q16]);
-                PF_LAP(6);
-                if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
-                cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_V16 + b1]);
-                PF_LAP(7);
-            }
-        }
-        PF_LAP_FLUSH(1);
-    } else if (warp < 12) {
-        // ------------------------------------------------ out: flow -> ring -----------------------------------
-        const int i = tid - 256;
-        const uint8_t* sQ = smem + F_Q;
-#pragma unroll 1
-        for (int k = 0; k < nk; ++k) {
-            const int b = k & 1;
-            int seq, c;
-            item(k, seq, c);
-            const int Cv = min(C, g.L - c * C);
-            uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
-            // ---- column i of Q (fp16) into registers, so that the Q buffer can take the next chunk early
-            if (!PF_WAIT(B_Q16, k & 1, 122)) return;
-            uint32_t qreg[32];
-            {
-                const uint8_t* qcol = sQ + (i >> 6) * 8192 + (i & 7) * 2;
-                const int ci = (i & 63) >> 3;
-#pragma unroll
-                for (int t = 0; t < 64; t += 2) {
-                    const uint32_t lo = *(const uint16_t*)(qcol + t * 128 + ((ci ^ (t & 7)) << 4));
-                    const uint32_t hi = *(const uint16_t*)(qcol + (t + 1) * 128 + ((ci ^ ((t + 1) & 7)) << 4));
-                    qreg[t >> 1] = lo | (hi << 16);
-                }
-            }
-            mbar_arrive(&bar[B_QCOPIED]);
-            PF_LAP(0);
-            bool ok = PF_WAIT(B_SLOTOK, k & 1, 121);      // the ring slot may be written
-            ok = ok && PF_WAIT(B_D34DONE, k & 1, 123);
+            PF_LAP(2);
+            // ---- RA = [E | Xi^T], first half: row i of E, one 16-byte piece per column group, into the ring
+            if (!PF_WAIT(B_SLOTOK, k & 1, 121) || !PF_WAIT(B_RADONE, k & 1, 123)) return;
             tc_fence_after();
-            if (!ok) return;
-            PF_LAP(1);
-            // ---- [E | Xi^T] from RA: row i of E and row j = i of Xi^T, one 16-byte piece per column group
+            PF_LAP(3);
             {
                 uint8_t* erow = slot + SLOT_E + i * 16;
-                uint8_t* xrow = slot + SLOT_XI + i * 16;
 #pragma unroll 1
-                for (int c0 = 0; c0 < DK + DV; c0 += 32) {
+                for (int c0 = 0; c0 < DK; c0 += 32) {
                     uint32_t rr[32];
                     tmem_ld32(RA + lane_base + c0, rr);
                     tmem_ld_wait();
-                    uint8_t* dst = (c0 < DK) ? erow + (c0 >> 3) * 2048 : xrow + ((c0 - DK) >> 3) * 2048;
 #pragma unroll
-                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(dst + j8 * 2048) = pack8(rr + 8 * j8, 1.f);
+                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(erow + ((c0 >> 3) + j8) * 2048) = pack8(rr + 8 * j8, 1.f);
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
-            PF_LAP(2);
-            // ---- Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t]: row i of the Qt image, straight into the ring
+            PF_LAP(4);
+            // ---- RB: Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t] (row i of the Qt image) and OI^T[j][t] -> OI[t][j] (fp32)
+            if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
+            tc_fence_after();
+            PF_LAP(5);
             {
                 uint8_t* qrow = slot + SLOT_QT + i * 16;
 #pragma unroll
@@ -578,10 +611,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                         *(uint4*)(qrow + ((c0 >> 3) + j8) * 2048) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
                 }
-            }
-            PF_LAP(3);
-            // ---- OI^T[j][t] -> OI[t][j] (fp32), straight into the ring
-            {
                 float* oi = (float*)(slot + SLOT_OI) + i;
 #pragma unroll 1
                 for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -597,7 +626,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_before();
             mbar_arrive(&bar[B_D4FREE]);
             mbar_arrive(&bar[B_OUTDONE]);
-            PF_LAP(4);
+            PF_LAP(6);
+            // ---- Q of the next chunk: convert in place, then take this thread's column
+            if (k + 1 < nk && !q_prepare(k + 1)) return;
+            PF_LAP(7);
         }
         PF_LAP_FLUSH(2);
     } else if (warp == 12) {
@@ -609,7 +641,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 int seq, c;
                 item(j, seq, c);
                 // K and V: their regions were last read by the MMAs of chunk j-2
-                if (j >= 2 && !PF_WAIT(B_D34DONE, (j - 2) & 1, 131)) return;
+                if (j >= 2 && !PF_WAIT(B_D4DONE, (j - 2) & 1, 131)) return;
                 mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
                 for (int h = 0; h < 2; ++h)
                     tma_load_3d(smem + b * F_REGION + K_OFF + h * KV_SLAB, &maps.k, 64 * h, c * C * r, seq, &bar[B_KFULL + b]);
@@ -669,6 +701,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 PF_LAP(4);
                 gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
                 gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
+                commit_uni(&bar[B_RADONE]);
                 // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T   (RB: G of chunk k+1 must have been drained)
                 if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
                 PF_LAP(5);
@@ -677,7 +710,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 PF_LAP(6);
                 gemm_uni<true, true, 64, N, N, N>(RB, x_b, pt_b);
                 gemm_uni<true, true, 64, N, N, N>(RB + 64, v_b, pt_b);
-                commit_uni(&bar[B_D34DONE]);
+                commit_uni(&bar[B_D4DONE]);
                 PF_LAP(7);
             }
             PF_LAP_FLUSH(4);
@@ -728,6 +761,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
     const int* ready = ws.ready + seq * g.R;
     volatile int* vis = (volatile int*)(smem + F_BAR + B_COUNT * 8 + 8);   // chunks whose ready flag the producer has acquired
+    volatile int* odone = (volatile int*)(smem + F_BAR + B_COUNT * 8 + 12); // output-warp completions (4 per chunk)
 
     if (warp < 8) {
         // ------------------------------------------------ chain: the state lives here -------------------------
@@ -842,7 +876,8 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             }
             tc_fence_before();
             mbar_arrive(&bar[B_OFREE + ob]);
-            mbar_arrive(&bar[B_ORPT + ob]);
+            __syncwarp();
+            if (lane == 0) atomicAdd((int*)odone, 1);       // (a counter, not a barrier: the reporter may lag by any amount)
             PF_LAP(1);
             if (c + 1 < NC && !fetch_oi(c + 1)) return;
             PF_LAP(2);
@@ -883,15 +918,28 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
         }
     } else if (warp == 13) {
         // ------------------------------------------------ consumed reports ------------------------------------
-        // Once the output warps are done with chunk c, chunks < c are consumed (the chain finished chunk c-1
-        // before it published the state for chunk c) and their ring slots may be rewritten.
+        // Once the four output warps are done with chunk c, chunks < c are consumed (the chain finished chunk c-1
+        // before it published the state for chunk c) and their ring slots may be rewritten.  The warp polls a
+        // shared counter and always reports the latest value, however far it has fallen behind.
         if (lane == 0) {
-#pragma unroll 1
-            for (int c = 0; c < NC; ++c) {
-                if (!PF_WAIT(B_ORPT + (c & 1), (c >> 1) & 1, 232)) return;
-                PF_LAP(0);
-                st_release_gpu(&ws.consumed[seq], c);
-                PF_LAP(1);
+            int reported = 0;
+            const long long t0 = clock64();
+            long long t_last = t0;
+            while (reported < NC - 1) {
+                const int chunks_done = *odone >> 2;
+                if (chunks_done - 1 > reported) {
+                    reported = chunks_done - 1;
+                    __threadfence_block();
+                    st_release_gpu(&ws.consumed[seq], reported);
+                    t_last = clock64();
+                } else if (clock64() - t_last > WAIT_CYCLES) {
+                    atomicCAS(err, 0, 232);
+                    break;
+                } else if (*(volatile int*)err != 0) {
+                    break;
+                } else {
+                    __nanosleep(200);
+                }
             }
             PF_LAP_FLUSH(12);
         }
@@ -922,7 +970,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
                 mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
                 mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
-                mbar_init(&bar[B_ORPT + x], 128); mbar_init(&bar[B_S16FREE + x], 1);
+                mbar_init(&bar[B_S16FREE + x], 1);
                 mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
             }
         } else {
@@ -933,16 +981,17 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
             }
             mbar_init(&bar[B_QFULL], 1); mbar_init(&bar[B_Q16], 128);
             mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128);
-            mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 128);
+            mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 256);
             mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 128);
-            mbar_init(&bar[B_D34DONE], 1); mbar_init(&bar[B_D4FREE], 128); mbar_init(&bar[B_RAFREE], 128);
-            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_OUTDONE], 128);
+            mbar_init(&bar[B_D4DONE], 1); mbar_init(&bar[B_RADONE], 1); mbar_init(&bar[B_D4FREE], 128); mbar_init(&bar[B_RAFREE], 256);
+            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_OUTDONE], 256);
             mbar_init(&bar[B_SLOTOK], 1);
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.v);
         }
         *(volatile int*)(smem + F_BAR + B_COUNT * 8 + 8) = 0;
+        *(volatile int*)(smem + F_BAR + B_COUNT * 8 + 12) = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base_s, 512);
