@@ -140,7 +140,8 @@ typedef struct pf_params {
 int pf_deltanet_fwd_ex(const pf_params* p);
 
 /* Bytes of scratch pf_deltanet_fwd_ex needs for this problem with this in_dtype/impl (0 on an
- * unsupported combination).  Host-only arithmetic; no CUDA call. */
+ * unsupported combination).  Host arithmetic; for the tensor-core implementations it asks the current
+ * device for its SM count (no allocation, no launch, no synchronisation). */
 size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
 
 /* Which PF_IMPL_* pf_deltanet_fwd_ex would run for this problem (negative pf_status if none). */

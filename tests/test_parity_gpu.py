@@ -208,3 +208,82 @@ def test_tc_full_path(w):
     """tc_flow + tc_scan: everything on tensor cores."""
     eo, es = _run_with_status(w, "tc")
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+# --- single-launch tensor-core path (flow builders and state scan side by side) -----------------------
+
+FUSED_CASES = [
+    Workload("fu_r2_c64", B=2, H=3, L=1000, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=41),       # n = 128, ring wraps
+    Workload("fu_r4_c32", B=1, H=2, L=333, d_k=128, d_v=128, r=4, chunk=32, beta_scale=2.0, s0_std=0.1, seed=42),
+    Workload("fu_r1_c64", B=2, H=2, L=700, d_k=128, d_v=128, r=1, chunk=64, s0_std=0.1, seed=43),       # n = 64
+    Workload("fu_r2_c32", B=1, H=3, L=450, d_k=128, d_v=128, r=2, chunk=32, seed=44),                   # n = 64, no S0
+    Workload("fu_r4_c16", B=1, H=2, L=130, d_k=128, d_v=128, r=4, chunk=16, beta_scale=2.0, seed=45),   # n = 64, C = 16
+    Workload("fu_short", B=3, H=1, L=17, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=46),         # less than a chunk
+    Workload("fu_many_seq", B=5, H=28, L=192, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=47),    # 140 scan CTAs, 8 flow CTAs
+]
+
+
+@pytest.mark.parametrize("w", FUSED_CASES, ids=lambda w: w.name)
+def test_fused_path_against_oracle(w):
+    eo, es = _run_with_status(w, "tc")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_fused_and_split_agree_and_ring_depth_is_invisible():
+    """The single-launch and the two-launch forms compute the same chunk algebra (different accumulation
+    orders and operand roundings: they agree to the bf16 tolerance); the ring depth changes only the
+    schedule, so results are bitwise identical across depths and across repeated runs."""
+    import paper_2504_00492_b200 as pf
+    w = Workload("fu_vs_split", B=2, H=2, L=1500, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=48)
+    d = pf_synth.make_inputs(w).to("cuda")
+    try:
+        outs = []
+        for depth in (3, 5, 8, 8, 21):
+            pf.pf_set_option("ring_depth", depth)
+            O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
+            torch.cuda.synchronize()
+            outs.append((O.clone(), Sf.clone()))
+    finally:
+        pf.pf_set_option("ring_depth", 8)
+    for O, Sf in outs[1:]:
+        assert torch.equal(O, outs[0][0]) and torch.equal(Sf, outs[0][1])
+    O2, S2 = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc_split")
+    assert util.max_rel(outs[0][0].cpu().numpy(), O2.cpu().numpy()) <= util.TOL_BF16
+    assert util.max_rel(outs[0][1].cpu().numpy(), S2.cpu().numpy()) <= util.TOL_BF16
+
+
+def test_too_many_sequences_take_the_two_launch_form():
+    """More sequences than scan CTAs can be placed: PF_IMPL_TC still works (two launches)."""
+    w = Workload("fu_fallback", B=6, H=25, L=130, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=49)   # 150 sequences
+    eo, es = _run_with_status(w, "tc")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_set_option_rejects_bad_input():
+    import paper_2504_00492_b200 as pf
+    with pytest.raises(pf.PfError) as ei:
+        pf.pf_set_option("ring_depth", 2)
+    assert ei.value.status == -1
+    with pytest.raises(pf.PfError) as ei:
+        pf.pf_set_option("no_such_option", 1)
+    assert ei.value.status == -2
+
+
+def test_back_to_back_launches_without_synchronisation():
+    """Several calls queued on one stream with a shared caller workspace: flags are reset in stream order."""
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    w = Workload("fu_b2b", B=1, H=8, L=4096, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=50)
+    d = pf_synth.make_inputs(w).to("cuda")
+    need = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "tc")
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    first = None
+    for rep in range(6):
+        for _ in range(3):
+            O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc", workspace=ws)
+        torch.cuda.synchronize()
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        if first is None:
+            first = (O.clone(), Sf.clone())
+        else:
+            assert torch.equal(O, first[0]) and torch.equal(Sf, first[1])
