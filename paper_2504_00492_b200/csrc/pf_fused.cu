@@ -9,13 +9,14 @@
 //           W  = diag(beta) X K,   Uh = diag(beta) X V
 //           E  = -K^T W,  Xi^T = Uh^T K                              (the chunk flow of Proposition 2.1)
 //           Qt = Q - P W (stored transposed),  OI = P Uh,            P = (Q K^T) (.) Mincl
-//       and store (E, Qt, Xi, OI) into slot (chunk mod R) of the sequence's ring;
+//       and store (E, Qt, Xi^T) into slot (chunk mod R) of the sequence's ring, OI into the chunk's rows of O;
 //   scan CTAs (one per sequence) carry the state over the chunks,
-//           O^T = OI^T + S Qt^T,      S <- S + S E^T + Xi^T,
+//           O += S Qt^T,      S <- S + S E^T + Xi^T,
 //       reading each slot as soon as its flag is set and freeing it for the flow CTAs afterwards.
 //
-// The ring (R slots of 112 KB per sequence) is rewritten in place, so the hand-off never has to reach HBM:
-// the only compulsory HBM traffic is one read of q, k, v, beta and one write of O.
+// The ring (R slots of 80 KB per sequence) is rewritten in place, so the hand-off never has to reach HBM; the
+// rows of O that hold OI are updated by the scan a few chunk steps after the flow CTA wrote them, while they
+// are still in L2.  The only compulsory HBM traffic is one read of q, k, v, beta and one write of O.
 //
 // A flow CTA is software-pipelined over two chunks (15 warps):
 //   warps 0-3  "solve"  epilogue of G = K K^T (mask, column scaling, fp16) and the triangular inverse
@@ -24,8 +25,8 @@
 //   warp 12             TMA loads (K and V double-buffered, Q single)
 //   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
 //   warp 14             ring back-pressure and ready flags
-// Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi^T]; RB = [256,384) holds G of the NEXT
-// chunk and then [Qt^T | OI^T] of the current one; RC = [384,448) holds P0^T.
+// Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi^T]; RG = [256,384) holds G of the NEXT
+// chunk; RC = [384,448) holds P0^T and then Qt^T; RD = [448,512) holds OI^T.
 // G is formed from the bf16 tiles as they land (both operands raw); every other product has a derived fp16
 // operand, so K, V and Q are converted to fp16 in place, off the critical path.
 //
@@ -60,8 +61,7 @@ constexpr int DK = 128, DV = 128;
 constexpr uint32_t SLOT_E = 0;                          // E image : fp16 [16 groups i'/8][128 rows i][16 B]  (K-major A)
 constexpr uint32_t SLOT_QT = SLOT_E + DK * DK * 2;      // Qt image: fp16 [ 8 groups t/8 ][128 rows i][16 B]  (MN-major B)
 constexpr uint32_t SLOT_XI = SLOT_QT + DK * 128;        // Xi^T    : fp16 [16 groups i/8 ][128 rows j][16 B]
-constexpr uint32_t SLOT_OI = SLOT_XI + DK * DV * 2;     // OI      : fp32 [64 rows t][128 cols j]
-constexpr uint32_t SLOT_BYTES = SLOT_OI + 64 * DV * 4;  // 114688
+constexpr uint32_t SLOT_BYTES = SLOT_XI + DK * DV * 2;  // 81920
 
 struct FusedGeo {
     int L, r, C, NC, nseq, R;
@@ -114,7 +114,7 @@ enum {
     B_PTREADY = 17,   // mid: P^T in shared memory (RC drained)
     B_D4DONE = 18,    // mma: [Qt^T | OI^T] complete (and everything issued before it)
     B_RADONE = 29,    // mma: [E | Xi^T] complete
-    B_D4FREE = 19,    // out: RB drained
+    B_D4FREE = 19,    // out: RC (Qt^T) and RD (OI^T) drained
     B_RAFREE = 20,    // out: RA drained
     B_QCOPIED = 25,   // out: Q copied into registers
     B_OUTDONE = 27,   // out: the chunk's images are stored
@@ -274,8 +274,8 @@ __device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, 
 // =============================================================================================================
 template <int N>
 __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedWs& ws,
-                          const __nv_bfloat16* __restrict__ beta, uint8_t* smem, uint64_t* bar, uint32_t tb,
-                          int fid) {
+                          const __nv_bfloat16* __restrict__ beta, float* __restrict__ O, uint8_t* smem, uint64_t* bar,
+                          uint32_t tb, int fid) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = g.r, C = g.C, nseq = g.nseq;
     int* err = ws.status;
@@ -287,7 +287,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     (void)t_lap; (void)lapacc;
     const int nk = fid < g.items ? (g.items - fid + g.n_flow - 1) / g.n_flow : 0;
-    const uint32_t RA = tb, RB = tb + 256, RC = tb + 384;
+    const uint32_t RA = tb, RG = tb + 256, RC = tb + 384, RD = tb + 448;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     constexpr uint32_t KV_SLAB = N * 128;                 // bytes of one 64-column slab of K / V / W / Uh
     constexpr uint32_t K_BYTES = N * 256;
@@ -340,7 +340,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 uint32_t rr[32];
                 const bool live = c0 < 32 * (warp + 1);
                 if (live) {
-                    tmem_ld32(RB + lane_base + c0, rr);
+                    tmem_ld32(RG + lane_base + c0, rr);
                     tmem_ld_wait();
                 }
                 if (m < N) {
@@ -588,7 +588,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
             PF_LAP(4);
-            // ---- RB: Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t] (row i of the Qt image) and OI^T[j][t] -> OI[t][j] (fp32)
+            // ---- RC: Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t] (row i of the Qt image);  RD: OI^T[j][t] -> OI[t][j] (fp32)
             if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
             tc_fence_after();
             PF_LAP(5);
@@ -597,7 +597,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t rr[32];
-                    tmem_ld32(RB + lane_base + c0, rr);
+                    tmem_ld32(RC + lane_base + c0, rr);
                     tmem_ld_wait();
 #pragma unroll
                     for (int j8 = 0; j8 < 4; ++j8) {
@@ -611,11 +611,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                         *(uint4*)(qrow + ((c0 >> 3) + j8) * 2048) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
                 }
-                float* oi = (float*)(slot + SLOT_OI) + i;
+                float* oi = O + ((long long)seq * g.L + (long long)c * C) * DV + i;     // OI[t][j = i] into the rows of O
 #pragma unroll 1
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t rr[32];
-                    tmem_ld32(RB + lane_base + 64 + c0, rr);
+                    tmem_ld32(RD + lane_base + c0, rr);
                     tmem_ld_wait();
                     const int lim = Cv - c0;
 #pragma unroll
@@ -662,7 +662,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_after();
             {
                 const uint32_t k_b = smem_u32(smem + K_OFF);
-                gemm_uni<false, false, N, DK, N, N, true>(RB, k_b, k_b);     // G(0) = K K^T from the bf16 tile
+                gemm_uni<false, false, N, DK, N, N, true>(RG, k_b, k_b);     // G(0) = K K^T from the bf16 tile
                 commit_uni(&bar[B_GDONE]);
             }
 #pragma unroll 1
@@ -679,21 +679,21 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
                 commit_uni(&bar[B_D2DONE]);
                 PF_LAP(1);
-                // P0^T = K Q^T   (RC was drained before MMA4 of chunk k-1 was issued)
-                if (!PF_WAIT(B_Q16, k & 1, 148)) return;
-                tc_fence_after();
-                PF_LAP(2);
-                gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
-                commit_uni(&bar[B_P0DONE]);
-                // G of the next chunk, from its bf16 tile
+                // G of the next chunk, from its bf16 tile (RG: the solve warps have drained G of this chunk)
                 if (k + 1 < nk) {
                     if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
-                    if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
                     tc_fence_after();
                     const uint32_t k1_b = smem_u32(smem + b1 * F_REGION + K_OFF);
-                    gemm_uni<false, false, N, DK, N, N, true>(RB, k1_b, k1_b);
+                    gemm_uni<false, false, N, DK, N, N, true>(RG, k1_b, k1_b);
                     commit_uni(&bar[B_GDONE]);
                 }
+                PF_LAP(2);
+                // P0^T = K Q^T   (RC and RD: Qt^T and OI^T of chunk k-1 have been drained)
+                if (!PF_WAIT(B_Q16, k & 1, 148)) return;
+                if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
+                tc_fence_after();
+                gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
+                commit_uni(&bar[B_P0DONE]);
                 PF_LAP(3);
                 // E = K^T (-W)  (lanes i, columns i'),   Xi^T = Uh^T K  (lanes j, columns i)
                 if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
@@ -702,14 +702,13 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
                 gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
                 commit_uni(&bar[B_RADONE]);
-                // [Qt^T - Q^T | OI^T] = [-W | Uh]^T P^T   (RB: G of chunk k+1 must have been drained)
-                if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
+                // Qt^T - Q^T = (-W)^T P^T over P0^T (which the out warps have turned into P^T),  OI^T = Uh^T P^T
                 PF_LAP(5);
-                if (k + 1 < nk && !PF_WAIT(B_GFREE, (k + 1) & 1, 151)) return;
+                if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
                 tc_fence_after();
                 PF_LAP(6);
-                gemm_uni<true, true, 64, N, N, N>(RB, x_b, pt_b);
-                gemm_uni<true, true, 64, N, N, N>(RB + 64, v_b, pt_b);
+                gemm_uni<true, true, 64, N, N, N>(RC, x_b, pt_b);
+                gemm_uni<true, true, 64, N, N, N>(RD, v_b, pt_b);
                 commit_uni(&bar[B_D4DONE]);
                 PF_LAP(7);
             }
@@ -851,7 +850,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) return false;
             const int Cv = min(g.C, g.L - c * g.C);
-            const float* oi = (const float*)(ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_OI) + j;
+            const float* oi = O + ((long long)seq * g.L + (long long)c * g.C) * DV + j;     // OI, left there by the flow CTA
 #pragma unroll
             for (int t = 0; t < 64; ++t) a[t] = (t < Cv) ? ld_cg_f32(oi + t * DV) : 0.f;
             return true;
@@ -1006,7 +1005,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     const uint32_t tb = tmem_base_s;
 
     if (is_scan) scan_role(g, ws, S0, O, S_final, smem, bar, tb, (int)blockIdx.x);
-    else flow_role<N>(maps, g, ws, beta, smem, bar, tb, (int)blockIdx.x - g.n_scan);
+    else flow_role<N>(maps, g, ws, beta, O, smem, bar, tb, (int)blockIdx.x - g.n_scan);
 
 
     tc_fence_before();
