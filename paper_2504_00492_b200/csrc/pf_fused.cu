@@ -71,8 +71,8 @@ struct FusedGeo {
 
 struct FusedWs {
     int* status;        // word 0: first expired wait (0 = none)
-    int* ready;         // [nseq][R]: chunk index + 1 once the slot holds that chunk
-    int* consumed;      // [nseq]: number of leading chunks the scan no longer needs
+    int* ready;         // [nseq][64] (R <= 64 used): chunk index + 1 once the slot holds that chunk; 256 B per sequence
+    int* consumed;      // [nseq][32]: word 0 = number of leading chunks the scan no longer needs; 128 B per sequence
     uint8_t* ring;      // [nseq][R][SLOT_BYTES]
 };
 
@@ -723,13 +723,13 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 item(k, seq, c);
                 const int slot_i = c % g.R;
                 // the scan must be done with the chunk that used this slot before
-                if (c >= g.R && !flag_wait_ge(&ws.consumed[seq], c - g.R + 1, err, 161)) return;
+                if (c >= g.R && !flag_wait_ge(&ws.consumed[seq * 32], c - g.R + 1, err, 161)) return;
                 mbar_arrive(&bar[B_SLOTOK]);
                 PF_LAP(0);
                 if (!PF_WAIT(B_OUTDONE, k & 1, 163)) return;
                 PF_LAP(1);
                 __threadfence();
-                st_release_gpu(&ws.ready[seq * g.R + slot_i], c + 1);
+                st_release_gpu(&ws.ready[seq * 64 + slot_i], c + 1);
                 PF_LAP(2);
             }
             PF_LAP_FLUSH(5);
@@ -758,7 +758,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const uint32_t t_delta = tb, t_o = tb + 128, t_a = tb + 256;     // Delta | 2 x O^T | 2 x fp16 state
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
-    const int* ready = ws.ready + seq * g.R;
+    const int* ready = ws.ready + seq * 64;
     volatile int* vis = (volatile int*)(smem + F_BAR + B_COUNT * 8 + 8);   // chunks whose ready flag the producer has acquired
     volatile int* odone = (volatile int*)(smem + F_BAR + B_COUNT * 8 + 12); // output-warp completions (4 per chunk)
 
@@ -929,7 +929,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 if (chunks_done - 1 > reported) {
                     reported = chunks_done - 1;
                     __threadfence_block();
-                    st_release_gpu(&ws.consumed[seq], reported);
+                    st_release_gpu(&ws.consumed[seq * 32], reported);
                     t_last = clock64();
                 } else if (clock64() - t_last > WAIT_CYCLES) {
                     atomicCAS(err, 0, 232);
@@ -1068,8 +1068,8 @@ Carve carve(const Problem& p) {
     Carve c{};
     c.status = 0;
     c.ready = 4096;
-    c.consumed = c.ready + align_up(nseq * R * 4, 256);
-    c.flag_bytes = align_up(c.consumed + nseq * 4, 1024);
+    c.consumed = c.ready + nseq * 256;          // every sequence's flags in cache lines of their own
+    c.flag_bytes = align_up(c.consumed + nseq * 128, 1024);
     c.ring = c.flag_bytes;
     c.total = c.ring + nseq * R * SLOT_BYTES;
     return c;
