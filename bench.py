@@ -16,6 +16,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import datetime
 import statistics
 import subprocess
 import sys
@@ -84,13 +85,20 @@ def ncu_traffic(w):
 
 
 class ClockSampler:
-    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs.
 
-    def __init__(self, gpu_index: int):
+    The first query of a process initialises the management library, which can hold up kernel launches for tens
+    of milliseconds, so the sampler is started before the warm-up and `wait_first_sample` returns once it is
+    past that.  Samples carry a timestamp; the summary uses those inside [t_begin, t_end] (host clock) when
+    there are any and says so in `window`, else every sample taken since the warm-up began (the GPU is kept
+    busy with the same kernel from then on)."""
+    Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int, period_ms: int = 20):
         self.gpu = gpu_index
+        self.period_ms = period_ms
         self.proc = None
         self.path = None
 
@@ -99,16 +107,36 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                          "--format=csv,noheader,nounits", "-lms", str(self.period_ms)], stdout=f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def wait_first_sample(self, busy, limit_s: float = 10.0):
+        """Calls busy() (which launches GPU work) until the first sample has been written."""
+        if self.proc is None:
+            return
+        t0 = time.time()
+        while time.time() - t0 < limit_s:
+            busy()
+            try:
+                if os.path.getsize(self.path) > 0:
+                    return
+            except OSError:
+                return
+
+    @staticmethod
+    def _stamp(text: str):
+        try:
+            return datetime.datetime.strptime(text.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, t_begin: float = None, t_end: float = None) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": None}
         if self.proc is None:
             return out
-        time.sleep(0.15)
+        time.sleep(2.5 * self.period_ms * 1e-3)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -119,21 +147,21 @@ class ClockSampler:
             os.unlink(self.path)
         except Exception:
             return out
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        parsed = []
         for r in rows:
-            if len(r) < 9:
+            if len(r) < 10:
                 continue
             try:
-                sm.append(float(r[1]))
-                mx.append(float(r[2]))
+                parsed.append((self._stamp(r[0]), float(r[2]), float(r[3]),
+                               [nm for nm, val in zip(names, r[6:10]) if val.strip().lower() == "active"]))
             except ValueError:
                 continue
-            for nm, val in zip(names, r[5:9]):
-                if val.strip().lower() == "active":
-                    reasons.add(nm)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        inside = [x for x in parsed if x[0] is not None and t_begin is not None and t_begin <= x[0] <= t_end]
+        use, window = (inside, "timed region") if inside else (parsed, "warm-up and timed region")
+        if use:
+            out.update(sm_mhz=statistics.median(x[1] for x in use), sm_max_mhz=max(x[2] for x in use),
+                       reasons=sorted({nm for x in use for nm in x[3]}), samples=len(use), window=window)
         return out
 
 
@@ -207,8 +235,8 @@ def kernel_profile(pf, d, w, steps):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(pf_synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -254,21 +282,23 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
-    launches_per_step = pf.pf_last_launch_count()
-    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample(lambda: (step(), torch.cuda.synchronize()))
+    for _ in range(args.warmup):
+        step()
+    launches_per_step = pf.pf_last_launch_count()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
+    t_begin = time.time()
     ev[0].record(stream)
     for i in range(args.steps):
         step()
         ev[i + 1].record(stream)
     barrier()
-    clocks = sampler.stop() if rank == 0 else {}
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else {}
     total_ms = ev[0].elapsed_time(ev[-1])
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     if use_dist:
@@ -367,7 +397,7 @@ def main():
             "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_k": w.d_k, "d_v": w.d_v, "r": w.r,
                        "chunk": w.chunk, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
                            (host.nbytes() + O.numel() * 4) / 1e6), "parallelism": "replicas" if world > 1 else "1 GPU"},
-            "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
             "token_heads_per_s": value * w.H,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},

@@ -36,9 +36,9 @@
 //
 // A scan CTA: warps 0-7 own the state (row j of S per thread, d_k split in two halves of 64 columns).  Each
 // chunk they write an fp16 copy of it into TENSOR memory, where it is the A operand of both of the chunk's
-// products (Delta = S E^T and O^T = S Qt^T, issued by warp 0), so the serial step never goes through shared
-// memory.  Warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt images in with bulk copies and is
-// the only poller of the ready flags, warp 13 reports consumed chunks.
+// products (Delta = S E^T issued by warp 0, O^T = S Qt^T issued by warp 13), so the serial step never goes
+// through shared memory.  Warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt images in with bulk
+// copies and is the only poller of the ready flags, warp 14 reports consumed chunks.
 //
 // Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
 // deliberately kept rolled: the instruction footprint of fifteen differently-specialised warps matters.
@@ -93,7 +93,8 @@ constexpr int SMEM_BYTES = F_BAR + 512;         // 230912
 constexpr int S_E = 0;                          // 2 x 32 KB  E images
 constexpr int S_XI = S_E + 2 * 32768;           // 2 x 32 KB  Xi images
 constexpr int S_QT = S_XI + 2 * 32768;          // 2 x 16 KB  Qt images
-static_assert(S_QT + 2 * 16384 <= F_BAR, "scan role fits below the barrier block");
+constexpr int S_OUT = S_QT + 2 * 16384;         // 2 x 32 KB  fp32 images of S Qt^T, [t][j], on their way into O
+static_assert(S_OUT + 2 * 32768 <= F_BAR, "scan role fits below the barrier block");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // barriers (indices into the uint64_t block at F_BAR)
@@ -126,6 +127,7 @@ enum {
     B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
+    B_APUB = 44,      // [2 buffers] mma: Delta of the chunk complete (the O^T product may be issued)
     B_S16FREE = 46,   // [2 buffers] mma: the MMAs that read that fp16 copy of the state are complete
     B_DDONE = 48,     // Delta complete
     B_ODONE = 50,     // [2] mma: O^T complete
@@ -161,6 +163,19 @@ __device__ __forceinline__ unsigned long long* timing_slot(const FusedWs& ws, bo
 #else
 #define PF_LAP(id) do { } while (0)
 #define PF_LAP_FLUSH(role) do { } while (0)
+#endif
+// Diagnostic builds (-DPF_STAMPS): the clock at each event of scan step PF_STAMP_STEP of sequence 0, written by
+// whole warps (no divergence) into unused shared memory of the scan role and copied to words 320.. of the
+// timing block when the chain ends: the timeline of one step.
+#ifdef PF_STAMPS
+#define PF_STAMP_STEP 64
+#define PF_STAMP_OFF (S_OUT + 2 * 32768)
+#define PF_STAMP(id)                                                                                       \
+    do {                                                                                                   \
+        if (seq == 0 && c == PF_STAMP_STEP) ((volatile uint32_t*)(smem + PF_STAMP_OFF))[(id)] = (uint32_t)clock64(); \
+    } while (0)
+#else
+#define PF_STAMP(id) do { } while (0)
 #endif
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
@@ -775,9 +790,11 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             const int buf = c & 1;
             // fp16 copy of the state into tensor memory (A operand of Delta and of O^T): 32 packed columns per thread
             bool ok = true;
+            PF_STAMP(0 + 10 * w);
             if (c >= 2) ok = PF_WAIT(B_S16FREE + buf, ((c >> 1) - 1) & 1, 201);
             tc_fence_after();
             PF_LAP(0);
+            PF_STAMP(1 + 10 * w);
             {
                 uint32_t pk[32];
 #pragma unroll
@@ -789,28 +806,27 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             tc_fence_before();
             if (!named_bar_and(1, 256, ok)) return;
             PF_LAP(2);
-            // warp 0 issues both products that read this copy of the state:
-            //   Delta[j][i] = sum_i' S[j][i'] E[i][i']   and   O^T[j][t] = sum_i S[j][i] Qt^T[i][t]
+            PF_STAMP(2 + 10 * w);
+            // warp 0 issues Delta[j][i] = sum_i' S[j][i'] E[i][i']; its completion also releases warp 13, which
+            // issues the O^T product of the same copy (so that O^T never sits in front of Delta in the tensor pipe)
             if (warp == 0) {
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
+                PF_STAMP(3);
                 gemm_ta<L_NSK, DK, DK, 128>(t_delta, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
-                if (!PF_WAIT(B_QTFULL + buf, (c >> 1) & 1, 234)) return;
-                if (c >= 2 && !PF_WAIT(B_OFREE + buf, ((c >> 1) - 1) & 1, 233)) return;
-                tc_fence_after();
-                gemm_ta<L_NSMN, 64, DK, 128>(t_o + buf * 64, t_a + buf * 64, smem_u32(smem + S_QT + buf * 16384));
-                commit_uni(&bar[B_ODONE + buf]);
-                commit_uni(&bar[B_QTEMPTY + buf]);
-                commit_uni(&bar[B_S16FREE + buf]);
+                commit_uni(&bar[B_APUB + buf]);
             }
             PF_LAP(3);
+            PF_STAMP(4 + 10 * w);
             if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
             PF_LAP(4);
+            PF_STAMP(5 + 10 * w);
             if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
             PF_LAP(5);
+            PF_STAMP(6 + 10 * w);
             // S += Delta + Xi^T   (row j, columns 64w..64w+63; Xi^T from its column-group image)
             const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + j * 16;
 #pragma unroll
@@ -833,64 +849,70 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
             PF_LAP(6);
+            PF_STAMP(7 + 10 * w);
         }
         PF_LAP_FLUSH(8 + w);
+#ifdef PF_STAMPS
+        if (seq == 0 && tid == 0)
+            for (int i_ = 0; i_ < 48; ++i_)
+                ((unsigned long long*)(ws.status + 256))[320 + i_] = ((volatile uint32_t*)(smem + PF_STAMP_OFF))[i_];
+#endif
         if (S_final)
 #pragma unroll
             for (int ii = 0; ii < 64; ++ii) S_final[sbase + (long long)ii * DV] = S[ii];
     } else if (warp < 12) {
-        // ------------------------------------------------ output: O^T = OI^T + S Qt^T --------------------------
-        // OI of the next chunk is fetched (into registers) while this chunk's MMA is awaited.
+        // ------------------------------------------------ output: O = OI + (S Qt^T)^T ---------------------------
+        // OI is already in the rows of O (left there by the flow CTA, visible once the chunk's ready flag has been
+        // acquired).  The chunk's S Qt^T goes from tensor memory into a [t][j] fp32 image in shared memory, which
+        // is exactly the layout of the chunk's rows of O, and one bulk reduction adds the image to them at the L2:
+        // OI is never read back, and the only per-thread work is the transposing copy.
         const int j = tid - 256;
-        float a[64];
-        auto fetch_oi = [&](int c) -> bool {
-            // (the producer warp has acquired the chunk's ready flag once *vis > c)
-            int ok = 1;
-            if (lane == 0) ok = smem_wait_ge(vis, c + 1, err, 211) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) return false;
-            const int Cv = min(g.C, g.L - c * g.C);
-            const float* oi = O + ((long long)seq * g.L + (long long)c * g.C) * DV + j;     // OI, left there by the flow CTA
-#pragma unroll
-            for (int t = 0; t < 64; ++t) a[t] = (t < Cv) ? ld_cg_f32(oi + t * DV) : 0.f;
-            return true;
-        };
 #pragma unroll 1
         for (int c = 0; c < NC; ++c) {
             const int ob = c & 1;
             const int Cv = min(g.C, g.L - c * g.C);
-            if (c == 0 && !fetch_oi(0)) return;
-            float* orow = O + ((long long)seq * g.L + (long long)c * g.C) * DV + j;
-            if (!PF_WAIT(B_ODONE + ob, (c >> 1) & 1, 212)) return;
+            float* img = (float*)(smem + S_OUT + ob * 32768);
+            PF_STAMP(20);
+            bool ok = PF_WAIT(B_ODONE + ob, (c >> 1) & 1, 212);
             tc_fence_after();
+            // the reduction of chunk c-2 has read this image (its issuing thread waits, the rest learn of it here)
+            if (tid == 256) {
+                bulk_wait_read_1();
+                ok = ok && smem_wait_ge(vis, c + 1, err, 211);     // (long since true: Qt was loaded after it)
+            }
+            if (!named_bar_and(2, 128, ok)) break;      // (every thread of the four warps leaves together)
             PF_LAP(0);
+            PF_STAMP(21);
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(t_o + ob * 64 + lane_base + c0, rr);
                 tmem_ld_wait();
 #pragma unroll
-                for (int t = 0; t < 32; ++t)
-                    if (c0 + t < Cv) orow[(long long)(c0 + t) * DV] = a[c0 + t] + __uint_as_float(rr[t]);
+                for (int t = 0; t < 32; ++t) img[(c0 + t) * DV + j] = __uint_as_float(rr[t]);
             }
             tc_fence_before();
             mbar_arrive(&bar[B_OFREE + ob]);
-            __syncwarp();
-            if (lane == 0) atomicAdd((int*)odone, 1);       // (a counter, not a barrier: the reporter may lag by any amount)
+            fence_async_smem();
+            named_bar(2, 128);
+            if (tid == 256) {
+                fence_async_global();
+                bulk_reduce_add_f32(O + ((long long)seq * g.L + (long long)c * g.C) * DV, img, (uint32_t)Cv * DV * 4u);
+                bulk_commit();
+                atomicAdd((int*)odone, 4);       // (a counter, not a barrier: the reporter may lag by any amount)
+            }
             PF_LAP(1);
-            if (c + 1 < NC && !fetch_oi(c + 1)) return;
-            PF_LAP(2);
+            PF_STAMP(22);
         }
+        if (tid == 256) bulk_wait_all();
         PF_LAP_FLUSH(10);
     } else if (warp == 12) {
         // ------------------------------------------------ producer: ring -> shared memory ----------------------
         if (lane == 0) {
             auto load_e = [&](int c) -> bool {
                 const int st = c & 1;
-                if (!flag_wait_ge(&ready[c % g.R], c + 1, err, 222)) return false;
+                if (!smem_wait_ge(vis, c + 1, err, 222)) return false;      // (warp 14 polls the ready flags, ahead of the loads)
                 fence_async_global();
-                __threadfence_block();
-                *vis = c + 1;
                 if (c >= 2 && !PF_WAIT(B_EEMPTY + st, ((c >> 1) - 1) & 1, 221)) return false;
                 mbar_expect_tx(&bar[B_EFULL + st], DK * DK * 2);
                 bulk_load(smem + S_E + st * 32768, ring + (size_t)(c % g.R) * SLOT_BYTES + SLOT_E, DK * DK * 2, &bar[B_EFULL + st]);
@@ -902,41 +924,77 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 // (the flag of chunk c was acquired by load_e(c))
                 const uint8_t* slot = ring + (size_t)(c % g.R) * SLOT_BYTES;
                 const int b = c & 1;
+                PF_STAMP(30);
                 if (c >= 2 && !PF_WAIT(B_XIEMPTY + b, ((c >> 1) - 1) & 1, 224)) return;
+                PF_STAMP(31);
                 mbar_expect_tx(&bar[B_XIFULL + b], DK * DV * 2);
                 bulk_load(smem + S_XI + b * 32768, slot + SLOT_XI, DK * DV * 2, &bar[B_XIFULL + b]);
                 PF_LAP(0);
                 if (c >= 2 && !PF_WAIT(B_QTEMPTY + b, ((c >> 1) - 1) & 1, 223)) return;
+                PF_STAMP(32);
                 mbar_expect_tx(&bar[B_QTFULL + b], DK * 128);
                 bulk_load(smem + S_QT + b * 16384, slot + SLOT_QT, DK * 128, &bar[B_QTFULL + b]);
                 PF_LAP(1);
                 if (c + 1 < NC && !load_e(c + 1)) return;
                 PF_LAP(2);
+                PF_STAMP(33);
             }
             PF_LAP_FLUSH(11);
         }
     } else if (warp == 13) {
-        // ------------------------------------------------ consumed reports ------------------------------------
-        // Once the four output warps are done with chunk c, chunks < c are consumed (the chain finished chunk c-1
-        // before it published the state for chunk c) and their ring slots may be rewritten.  The warp polls a
-        // shared counter and always reports the latest value, however far it has fallen behind.
+        // ------------------------------------------------ O^T[j][t] = sum_i S[j][i] Qt^T[i][t] (whole warp) -----
+#pragma unroll 1
+        for (int c = 0; c < NC; ++c) {
+            const int buf = c & 1;
+            PF_STAMP(40);
+            if (!PF_WAIT(B_APUB + buf, (c >> 1) & 1, 235)) return;
+            PF_STAMP(41);
+            if (!PF_WAIT(B_QTFULL + buf, (c >> 1) & 1, 234)) return;
+            PF_STAMP(42);
+            if (c >= 2 && !PF_WAIT(B_OFREE + buf, ((c >> 1) - 1) & 1, 233)) return;
+            PF_STAMP(43);
+            tc_fence_after();
+            gemm_ta<L_NSMN, 64, DK, 128>(t_o + buf * 64, t_a + buf * 64, smem_u32(smem + S_QT + buf * 16384));
+            commit_uni(&bar[B_ODONE + buf]);
+            commit_uni(&bar[B_QTEMPTY + buf]);
+            commit_uni(&bar[B_S16FREE + buf]);
+            PF_STAMP(44);
+        }
+    } else {
+        // ------------------------------------------------ ready flags in, consumed reports out -----------------
+        // One lane polls the ring's ready flags in chunk order, as far ahead of the loads as the flow CTAs are, and
+        // publishes the count in shared memory (so that no load waits a trip to the L2 for a flag that was set long
+        // ago).  The same loop reports consumption: once the four output warps are done with chunk c, chunks < c
+        // are consumed (the chain finished chunk c-1 before it published the state for chunk c) and their ring
+        // slots may be rewritten.  It polls a shared counter and always reports the latest value, however far it
+        // has fallen behind.
         if (lane == 0) {
-            int reported = 0;
+            int reported = 0, seen = 0;
             const long long t0 = clock64();
             long long t_last = t0;
-            while (reported < NC - 1) {
+            while (reported < NC - 1 || seen < NC) {
+                bool progress = false;
+                if (seen < NC && ld_acquire_gpu(&ready[seen % g.R]) >= seen + 1) {
+                    ++seen;
+                    __threadfence_block();
+                    *vis = seen;
+                    progress = true;
+                }
                 const int chunks_done = *odone >> 2;
                 if (chunks_done - 1 > reported) {
                     reported = chunks_done - 1;
                     __threadfence_block();
                     st_release_gpu(&ws.consumed[seq * 32], reported);
+                    progress = true;
+                }
+                if (progress) {
                     t_last = clock64();
                 } else if (clock64() - t_last > WAIT_CYCLES) {
                     atomicCAS(err, 0, 232);
                     break;
                 } else if (*(volatile int*)err != 0) {
                     break;
-                } else {
+                } else if (seen == NC) {
                     __nanosleep(200);
                 }
             }
@@ -969,7 +1027,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
                 mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
                 mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
-                mbar_init(&bar[B_S16FREE + x], 1);
+                mbar_init(&bar[B_APUB + x], 1); mbar_init(&bar[B_S16FREE + x], 1);
                 mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
             }
         } else {
