@@ -38,10 +38,10 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build())
-        fn = lib.pf_oracle_deltanet_fwd_f64
-        fn.restype = ctypes.c_int
-        fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int] * 6 + [ctypes.c_void_p] * 2 + [
-            ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+        for fn in (lib.pf_oracle_deltanet_fwd_f64, lib.pf_oracle_deltanet_product_fwd_f64):
+            fn.restype = ctypes.c_int
+            fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int] * 6 + [ctypes.c_void_p] * 2 + [
+                ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         _lib = lib
     return _lib
 
@@ -66,8 +66,9 @@ def _to_numpy(x):
     return np.asarray(x)
 
 
-def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: bool = False):
-    """Run the recurrence.  Shapes: q [B,H,L,d_k], k [B,H,L,r,d_k], v [B,H,L,r,d_v], beta [B,H,L,r],
+def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: bool = False, mode: str = "sum"):
+    """Run the recurrence.  ``mode``: "sum" (all r factors of a token read the same old state: the paper's
+    rank-R form) or "product" (the factors act one after another: rank-1 delta rule r times per token).  Shapes: q [B,H,L,d_k], k [B,H,L,r,d_k], v [B,H,L,r,d_v], beta [B,H,L,r],
     S0 [B,H,d_k,d_v] or None.  Inputs may be numpy or torch (bf16/fp16/fp32); they are widened
     exactly, the arithmetic is fp64.  Returns (O [B,H,L,d_v] float64, S_final [B,H,d_k,d_v] float64)
     and, if ``return_threads``, the number of host threads used."""
@@ -88,7 +89,10 @@ def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: b
     O = np.empty((B, H, L, d_v), dtype=np.float64)
     Sf = np.empty((B, H, d_k, d_v), dtype=np.float64)
     used = ctypes.c_int(0)
-    rc = _load().pf_oracle_deltanet_fwd_f64(
+    if mode not in ("sum", "product"):
+        raise ValueError("mode must be 'sum' or 'product'")
+    fn = _load().pf_oracle_deltanet_fwd_f64 if mode == "sum" else _load().pf_oracle_deltanet_product_fwd_f64
+    rc = fn(
         qa.ctypes.data, ka.ctypes.data, va.ctypes.data, ba.ctypes.data,
         s0.ctypes.data if s0 is not None else None,
         B, H, L, d_k, d_v, r, O.ctypes.data, Sf.ctypes.data, int(num_threads), ctypes.byref(used))

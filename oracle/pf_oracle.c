@@ -19,6 +19,16 @@
  * above.  All r factors of a token read the SAME old state (diagonal R x R blocks of
  * Id - M (.) A B^T are the identity, proof of Theorem 3.2), i.e. the "sum" form.
  *
+ * A second entry point evaluates the PRODUCT form, in which the r factors of a token act one after
+ * another, each on the state the previous one left:
+ *
+ *     S_t = S_{t-1} prod_j (I - beta_{t,j} k_{t,j} k_{t,j}^T)  + (the matching v terms),
+ *
+ * i.e. the rank-1 delta rule of Section 1.3 applied r times per token (the same thing as rank-1
+ * DeltaNet on the length L*r sequence of factors, read out after every r-th step).  In the chunk form
+ * of Theorem 3.2 this is the general block-triangular case, with the mask strict in the flattened
+ * row index instead of the time index.
+ *
  * Every pin that ties this file to something other than itself is in tests/test_oracle_pins.py.
  *
  * Layouts (all row-major, host memory):
@@ -85,12 +95,55 @@ static void pf_oracle_one_sequence(const float* q, const float* k, const float* 
                 S_final[(size_t)i * d_v + j] = S[(size_t)j * d_k + i];
 }
 
+/* One sequence, product form: factor f reads the state factor f-1 left (rank-1 delta rule, r times). */
+static void pf_oracle_one_sequence_product(const float* q, const float* k, const float* v, const float* beta,
+                                           const double* S0, int L, int d_k, int d_v, int r,
+                                           double* O, double* S_final, double* S, double* p)
+{
+    for (int j = 0; j < d_v; ++j)
+        for (int i = 0; i < d_k; ++i)
+            S[(size_t)j * d_k + i] = S0 ? S0[(size_t)i * d_v + j] : 0.0;
+
+    for (int t = 0; t < L; ++t) {
+        for (int f = 0; f < r; ++f) {
+            const float* kf = k + ((size_t)t * r + f) * d_k;
+            const float* vf = v + ((size_t)t * r + f) * d_v;
+            const double b = (double)beta[(size_t)t * r + f];
+            /* prediction from the CURRENT state, then S <- S + beta (v - S k) k^T */
+            for (int j = 0; j < d_v; ++j) {
+                double acc = 0.0;
+                for (int i = 0; i < d_k; ++i)
+                    acc += S[(size_t)j * d_k + i] * (double)kf[i];
+                p[j] = acc;
+            }
+            for (int j = 0; j < d_v; ++j) {
+                double e = b * ((double)vf[j] - p[j]);
+                for (int i = 0; i < d_k; ++i)
+                    S[(size_t)j * d_k + i] += e * (double)kf[i];
+            }
+        }
+        /* o_t = S_t q_t, after the token's last factor */
+        const float* qt = q + (size_t)t * d_k;
+        for (int j = 0; j < d_v; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < d_k; ++i)
+                acc += S[(size_t)j * d_k + i] * (double)qt[i];
+            O[(size_t)t * d_v + j] = acc;
+        }
+    }
+
+    if (S_final)
+        for (int j = 0; j < d_v; ++j)
+            for (int i = 0; i < d_k; ++i)
+                S_final[(size_t)i * d_v + j] = S[(size_t)j * d_k + i];
+}
+
 /* Returns 0 on success, -1 on a bad argument, -2 on allocation failure.
  * num_threads <= 0 means "whatever OpenMP picks"; sequences (b,h) are independent, and that is the
  * only parallelism used.  *threads_used (may be NULL) receives the thread count actually used. */
-int pf_oracle_deltanet_fwd_f64(const float* q, const float* k, const float* v, const float* beta,
-                               const double* S0, int B, int H, int L, int d_k, int d_v, int r,
-                               double* O, double* S_final, int num_threads, int* threads_used)
+static int pf_oracle_run(int product, const float* q, const float* k, const float* v, const float* beta,
+                         const double* S0, int B, int H, int L, int d_k, int d_v, int r,
+                         double* O, double* S_final, int num_threads, int* threads_used)
 {
     if (!q || !k || !v || !beta || !O) return -1;
     if (B < 1 || H < 1 || L < 0 || d_k < 1 || d_v < 1 || r < 1) return -1;
@@ -122,7 +175,8 @@ int pf_oracle_deltanet_fwd_f64(const float* q, const float* k, const float* v, c
 #pragma omp for schedule(dynamic, 1)
 #endif
             for (int s = 0; s < nseq; ++s) {
-                pf_oracle_one_sequence(q + (size_t)s * L * d_k,
+                (product ? pf_oracle_one_sequence_product : pf_oracle_one_sequence)(
+                                       q + (size_t)s * L * d_k,
                                        k + (size_t)s * L * r * d_k,
                                        v + (size_t)s * L * r * d_v,
                                        beta + (size_t)s * L * r,
@@ -137,4 +191,19 @@ int pf_oracle_deltanet_fwd_f64(const float* q, const float* k, const float* v, c
         free(p);
     }
     return failed ? -2 : 0;
+}
+
+int pf_oracle_deltanet_fwd_f64(const float* q, const float* k, const float* v, const float* beta,
+                               const double* S0, int B, int H, int L, int d_k, int d_v, int r,
+                               double* O, double* S_final, int num_threads, int* threads_used)
+{
+    return pf_oracle_run(0, q, k, v, beta, S0, B, H, L, d_k, d_v, r, O, S_final, num_threads, threads_used);
+}
+
+/* Product form (see the header): same arguments, same layouts, same return codes. */
+int pf_oracle_deltanet_product_fwd_f64(const float* q, const float* k, const float* v, const float* beta,
+                                       const double* S0, int B, int H, int L, int d_k, int d_v, int r,
+                                       double* O, double* S_final, int num_threads, int* threads_used)
+{
+    return pf_oracle_run(1, q, k, v, beta, S0, B, H, L, d_k, d_v, r, O, S_final, num_threads, threads_used);
 }

@@ -101,8 +101,10 @@ def interval_flow(k, v, beta):
     return P, Xi
 
 
-def chunked_forward(q, k, v, beta, S0, chunk):
+def chunked_forward(q, k, v, beta, S0, chunk, product=False):
     """The chunk-form forward pass for one sequence in fp64 (what the kernels compute, step by step).
+    ``product``: the strict mask is taken in the flattened row index m' < m instead of the time index
+    (the general block-triangular case: the factors of a token act one after another).
 
     q [L,d_k], k [L,r,d_k], v [L,r,d_v], beta [L,r], S0 [d_k,d_v] or None.
     Per chunk (rows m = t*r + j, n = C*r):
@@ -123,7 +125,9 @@ def chunked_forward(q, k, v, beta, S0, chunk):
         b = beta[c0:c1].reshape(n)
         Q = q[c0:c1]
         tok = np.arange(n) // r
-        Lm = np.eye(n) + (tok[None, :] < tok[:, None]) * (b[:, None] * (K @ K.T))
+        rows = np.arange(n)
+        strict = (rows[None, :] < rows[:, None]) if product else (tok[None, :] < tok[:, None])
+        Lm = np.eye(n) + strict * (b[:, None] * (K @ K.T))
         Tp = scipy.linalg.solve_triangular(Lm, np.diag(b), lower=True)
         W = Tp @ K
         Uh = Tp @ V

@@ -362,3 +362,91 @@ def test_empty_sequence_returns_S0():
     O, Sf = oracle.deltanet_fwd(q, k, v, beta, S0)
     assert O.shape == (1, 1, 0, 3)
     np.testing.assert_allclose(Sf, S0, rtol=0, atol=0)
+
+
+# --- product form: the r factors of a token act one after another -------------------------------------
+# (rank-1 delta rule of Section 1.3, r times per token; the chunk form is the general block-triangular case
+# of Theorem 3.2 with the mask strict in the flattened row index)
+
+def test_product_form_is_rank1_deltanet_on_the_interleaved_sequence():
+    # the sum-form oracle with r = 1 (pinned by everything above) on the L*r factors, read out every r-th step
+    L, r, d_k, d_v = 7, 3, 6, 5
+    q, k, v, beta, S0 = make(80, L=L, r=r, d_k=d_k, d_v=d_v, B=1, H=2, beta_hi=1.8)
+    O, Sf = oracle.deltanet_fwd(q, k, v, beta, S0, mode="product")
+    k1 = k.reshape(1, 2, L * r, 1, d_k)
+    v1 = v.reshape(1, 2, L * r, 1, d_v)
+    b1 = beta.reshape(1, 2, L * r, 1)
+    q1 = np.repeat(q, r, axis=2)
+    O1, Sf1 = oracle.deltanet_fwd(q1, k1, v1, b1, S0)
+    np.testing.assert_allclose(O, O1[:, :, r - 1::r], rtol=0, atol=TOL)
+    np.testing.assert_allclose(Sf, Sf1, rtol=0, atol=TOL)
+
+
+def test_product_form_brute_force_matrices():
+    # explicit d_k x d_k transition matrices, multiplied out in numpy
+    L, r, d_k, d_v = 5, 2, 4, 3
+    q, k, v, beta, S0 = make(81, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=1.9)
+    O, Sf = oracle.deltanet_fwd(q, k, v, beta, S0, mode="product")
+    qd, kd, vd, bd, s0 = f64(q[0, 0], k[0, 0], v[0, 0], beta[0, 0], S0[0, 0])
+    S = s0.T.copy()
+    for t in range(L):
+        for j in range(r):
+            kk, vv, b = kd[t, j], vd[t, j], bd[t, j]
+            S = S @ (np.eye(d_k) - b * np.outer(kk, kk)) + b * np.outer(vv, kk)
+        np.testing.assert_allclose(O[0, 0, t], S @ qd[t], rtol=0, atol=TOL)
+    np.testing.assert_allclose(Sf[0, 0], S.T, rtol=0, atol=TOL)
+
+
+def test_product_equals_sum_when_a_tokens_keys_are_orthogonal():
+    # (I - b1 k1 k1^T)(I - b2 k2 k2^T) = I - b1 k1 k1^T - b2 k2 k2^T  and  v1 k1^T (I - b2 k2 k2^T) = v1 k1^T
+    L, r, d_k, d_v = 6, 3, 8, 4
+    q, k, v, beta, S0 = make(82, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=1.5)
+    g = rnd(83)
+    for t in range(L):
+        Qm, _ = np.linalg.qr(g.standard_normal((d_k, d_k)))
+        k[0, 0, t] = Qm[:r].astype(np.float32)
+    # float32 rounding leaves the keys orthogonal only to ~1e-7: compare at that level
+    O_s, Sf_s = oracle.deltanet_fwd(q, k, v, beta, S0)
+    O_p, Sf_p = oracle.deltanet_fwd(q, k, v, beta, S0, mode="product")
+    np.testing.assert_allclose(O_p, O_s, rtol=0, atol=5e-6)
+    np.testing.assert_allclose(Sf_p, Sf_s, rtol=0, atol=5e-6)
+
+
+def test_product_form_depends_on_factor_order_and_r1_is_the_sum_form():
+    L, r, d_k, d_v = 6, 2, 5, 4
+    q, k, v, beta, S0 = make(84, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=1.5)
+    _, Sf = oracle.deltanet_fwd(q, k, v, beta, S0, mode="product")
+    _, Sf_swapped = oracle.deltanet_fwd(q, k[:, :, :, ::-1], v[:, :, :, ::-1], beta[:, :, :, ::-1], S0, mode="product")
+    assert np.abs(Sf - Sf_swapped).max() > 1e-3
+    _, Sf_sum = oracle.deltanet_fwd(q, k, v, beta, S0)
+    assert np.abs(Sf - Sf_sum).max() > 1e-3
+    O1, S1 = oracle.deltanet_fwd(q, k[:, :, :, :1], v[:, :, :, :1], beta[:, :, :, :1], S0)
+    O2, S2 = oracle.deltanet_fwd(q, k[:, :, :, :1], v[:, :, :, :1], beta[:, :, :, :1], S0, mode="product")
+    np.testing.assert_array_equal(O1, O2)
+    np.testing.assert_array_equal(S1, S2)
+
+
+def test_product_form_is_contractive_for_beta_in_0_2():
+    # unit keys, v = 0: every factor I - b k k^T has norm <= 1 for b in [0, 2], and is orthogonal for b = 2
+    L, r, d_k, d_v = 40, 3, 6, 5
+    q, k, v, beta, S0 = make(85, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=2.0)
+    k = unit(k)
+    v = np.zeros_like(v)
+    norms = [np.linalg.norm(f64(S0[0, 0])[0])]
+    for t in range(1, L + 1):
+        _, Sf = oracle.deltanet_fwd(q[:, :, :t], k[:, :, :t], v[:, :, :t], beta[:, :, :t], S0, mode="product")
+        norms.append(np.linalg.norm(Sf[0, 0]))
+    assert all(b <= a * (1 + 1e-6) for a, b in zip(norms, norms[1:]))
+    beta2 = np.full_like(beta, 2.0)
+    _, Sf2 = oracle.deltanet_fwd(q, k, v, beta2, S0, mode="product")
+    np.testing.assert_allclose(np.linalg.norm(Sf2[0, 0]), norms[0], rtol=1e-5)
+
+
+@pytest.mark.parametrize("L,r,d_k,d_v,chunk", [(37, 2, 6, 5, 8), (50, 3, 8, 8, 16), (16, 4, 4, 6, 16)])
+def test_chunk_form_with_flattened_mask_matches_product_recurrence(L, r, d_k, d_v, chunk):
+    q, k, v, beta, S0 = make(86, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=1.7)
+    O, Sf = oracle.deltanet_fwd(q, k, v, beta, S0, mode="product")
+    qd, kd, vd, bd, s0 = f64(q[0, 0], k[0, 0], v[0, 0], beta[0, 0], S0[0, 0])
+    O_c, Sf_c, _ = pfm.chunked_forward(qd, kd, vd, bd, s0, chunk, product=True)
+    np.testing.assert_allclose(O_c, O[0, 0], rtol=0, atol=1e-11)
+    np.testing.assert_allclose(Sf_c, Sf[0, 0], rtol=0, atol=1e-11)
