@@ -56,6 +56,20 @@ typedef enum pf_status {
 
 enum { PF_DTYPE_BF16 = 0, PF_DTYPE_F32 = 1 };
 
+/* How the r factors of one token combine (pf_params.mode).
+ *   PF_MODE_SUM     : all r factors read the same previous state,
+ *                         S_t = S_{t-1} (I - sum_j beta_j k_j k_j^T) + sum_j beta_j v_j k_j^T.
+ *                     This is the paper's rank-R form (Section 3.1; in the proof of Theorem 3.2 the
+ *                     diagonal R x R blocks of Id - M (.) A B^T are the identity) and what every entry
+ *                     point without a mode argument computes.
+ *   PF_MODE_PRODUCT : the factors act one after another, each on the state the previous one left,
+ *                         S_t = S_{t-1} prod_j (I - beta_j k_j k_j^T) + (the matching v terms),
+ *                     i.e. the rank-1 delta rule of Section 1.3 applied r times per token, read out after
+ *                     the token's last factor.  In the chunk form it is the general block-triangular
+ *                     case of Theorem 3.2: Mstrict[m,m'] = 1(m' < m) in the flattened row index; every
+ *                     other formula is unchanged.  Every factor is a contraction for beta in [0, 2]. */
+enum { PF_MODE_SUM = 0, PF_MODE_PRODUCT = 1 };
+
 /* Which kernels evaluate the chunk form.
  *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
@@ -132,6 +146,7 @@ typedef struct pf_params {
                                  or NULL: stream-ordered allocation inside the call */
     size_t workspace_bytes;
     void* stream;
+    int mode;                 /* PF_MODE_SUM (0) or PF_MODE_PRODUCT; anything else: PF_ERR_INVALID */
 } pf_params;
 
 /* Same operation with explicit options.  The workspace holds per-chunk intermediates (T', W, Uh, P

@@ -19,6 +19,8 @@ PF_DTYPE_BF16, PF_DTYPE_F32 = 0, 1
 PF_IMPL_AUTO, PF_IMPL_SIMT, PF_IMPL_TC = 0, 1, 2
 PF_IMPL_TC_REFFLOW = 3
 PF_IMPL_TC_SPLIT = 4
+PF_MODE_SUM, PF_MODE_PRODUCT = 0, 1
+MODE_BY_NAME = {"sum": PF_MODE_SUM, "product": PF_MODE_PRODUCT}
 IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC, "tc_refflow": PF_IMPL_TC_REFFLOW,
                 "tc_split": PF_IMPL_TC_SPLIT}
 
@@ -41,6 +43,7 @@ class PfParams(ctypes.Structure):
         ("in_dtype", ctypes.c_int), ("impl", ctypes.c_int),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p),
+        ("mode", ctypes.c_int),
     ]
 
 
@@ -182,9 +185,10 @@ def pf_static_scratch_bytes() -> int:
 
 
 def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Optional[torch.Tensor] = None,
-                       O=None, S_final=None, stream=None, want_state: bool = True):
+                       O=None, S_final=None, stream=None, want_state: bool = True, mode="sum"):
     """Same operation with an explicit implementation and (optionally) a caller-owned workspace
-    (a uint8 CUDA tensor of at least pf_workspace_bytes(...) bytes)."""
+    (a uint8 CUDA tensor of at least pf_workspace_bytes(...) bytes).  mode: "sum" (the r factors of a token
+    read the same previous state) or "product" (they act one after another)."""
     dtype = q.dtype
     if dtype not in (torch.bfloat16, torch.float32):
         raise TypeError("q/k/v/beta must be bf16 or fp32")
@@ -199,6 +203,7 @@ def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Op
     if workspace is not None:
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.stream = _stream(stream)
+    p.mode = MODE_BY_NAME[mode] if isinstance(mode, str) else int(mode)
     with torch.cuda.device(q.device):
         st = lib().pf_deltanet_fwd_ex(ctypes.byref(p))
     if st != 0:

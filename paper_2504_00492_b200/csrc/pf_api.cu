@@ -93,7 +93,9 @@ int forward(const pf_params* a) {
     if (!a) return PF_ERR_INVALID;
     int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
     if (st != PF_OK) return st;
+    if (a->mode != PF_MODE_SUM && a->mode != PF_MODE_PRODUCT) return PF_ERR_INVALID;
     Problem p = as_problem(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk, a->in_dtype);
+    p.mode = a->mode;
     const int impl = select_impl(p, a->impl);
     if (impl < 0) return impl;
     if (a->L > 0 && (!a->q || !a->k || !a->v || !a->beta || !a->O)) return PF_ERR_INVALID;

@@ -22,9 +22,13 @@ struct Problem {
     float* O;
     float* S_final;
     int in_dtype;
+    int mode;           // PF_MODE_SUM (0) or PF_MODE_PRODUCT
     cudaStream_t stream;
 
     __host__ __device__ int n() const { return chunk * r; }            // rows per chunk
+    // Rows m' < m of a chunk interact (the strict mask of Theorem 3.2) when they lie in different groups of this
+    // many consecutive rows: r for the sum form (different tokens), 1 for the product form (any earlier row).
+    __host__ __device__ int mask_group() const { return mode == PF_MODE_PRODUCT ? 1 : r; }
     __host__ __device__ int chunks_per_seq() const { return (L + chunk - 1) / chunk; }
     __host__ __device__ long long total_chunks() const { return (long long)B * H * chunks_per_seq(); }
 };

@@ -65,6 +65,7 @@ constexpr uint32_t SLOT_BYTES = SLOT_XI + DK * DV * 2;  // 81920
 
 struct FusedGeo {
     int L, r, C, NC, nseq, R;
+    int rm;             // strict-mask group size (Problem::mask_group)
     int n_scan, n_flow;
     int items;          // nseq * NC
 };
@@ -317,7 +318,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     if (warp < 4) {
         // ------------------------------------------------ solve: G epilogue + triangular inverse -------------
         const int m = tid;
-        const int row_lim = (m / r) * r;       // rows m' < row_lim belong to earlier tokens
+        const int row_lim = (m / g.rm) * g.rm; // rows m' < row_lim: earlier tokens (sum form) / earlier rows (product form)
         float* sBeta = (float*)(smem + F_BETA);
         float beta_next = 0.f;
         if (nk > 0) {
@@ -1170,7 +1171,7 @@ int fused_forward(const Problem& p, void* workspace) {
     ws.ring = base + cv.ring;
     PF_CUDA_TRY(cudaMemsetAsync(base, 0, cv.flag_bytes, p.stream));
     FusedGeo g{};
-    g.L = p.L; g.r = p.r; g.C = p.chunk; g.NC = NC; g.nseq = nseq; g.R = ring_depth(p);
+    g.L = p.L; g.r = p.r; g.C = p.chunk; g.NC = NC; g.nseq = nseq; g.R = ring_depth(p); g.rm = p.mask_group();
     g.items = nseq * NC;
     const int sms = sm_count();
     g.n_scan = nseq;

@@ -24,6 +24,7 @@ template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloa
 
 struct Geo {
     int L, d_k, d_v, r, C, n, NC;   // NC = chunks per sequence
+    int rm;                         // strict-mask group size (Problem::mask_group)
 };
 
 // Workspace (fp32), G = total chunks:  T [G][n][n]  W [G][n][d_k]  U [G][n][d_v]  P [G][C][n]
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(256) simt_gram(const Tin* __restrict__ q, cons
     float* Pg = ws.P + gc * (long long)g.C * n;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 
-    // A[m][m'] = beta_m (k_m . k_m') for tok(m') < tok(m), else 0
+    // A[m][m'] = beta_m (k_m . k_m') for tok(m') < tok(m) (product form: m' < m), else 0
     for (int m0 = 0; m0 < n; m0 += TM)
         for (int n0 = 0; n0 < n; n0 += 64) {
             float acc[4][4];
@@ -125,7 +126,7 @@ __global__ void __launch_bounds__(256) simt_gram(const Tin* __restrict__ q, cons
                 for (int j = 0; j < 4; ++j) {
                     const int mp = n0 + tx * 4 + j;
                     if (mp >= n) continue;
-                    Tg[(long long)m * n + mp] = (mp / r < m / r) ? bm * acc[i][j] : 0.f;
+                    Tg[(long long)m * n + mp] = (mp / g.rm < m / g.rm) ? bm * acc[i][j] : 0.f;
                 }
             }
         }
@@ -187,7 +188,7 @@ __global__ void simt_solve(const Tin* __restrict__ beta, Geo g, Ws ws) {
         for (int mm = 0; mm < RB; ++mm) {
             const int m = m0 + mm;
             if (m >= n || m < wstart) continue;      // whole warp above the diagonal
-            const int lim = (m / r) * r;             // rows of the same token do not interact
+            const int lim = (m / g.rm) * g.rm;       // rows of the same token do not interact (sum form)
             float acc = 0.f;
             for (int mp = wstart; mp < lim; ++mp) {
                 const float a = Ar[mm * n + mp];                              // broadcast
@@ -365,7 +366,7 @@ Ws carve(const Problem& p, void* workspace) {
 
 template <class Tin>
 int run(const Problem& p, void* workspace, bool prepare_only) {
-    Geo g{p.L, p.d_k, p.d_v, p.r, p.chunk, p.n(), p.chunks_per_seq()};
+    Geo g{p.L, p.d_k, p.d_v, p.r, p.chunk, p.n(), p.chunks_per_seq(), p.mask_group()};
     const long long G = p.total_chunks();
     const long long nseq = (long long)p.B * p.H;
     const Tin* q = (const Tin*)p.q;

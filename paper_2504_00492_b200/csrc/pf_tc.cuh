@@ -7,6 +7,7 @@ namespace pf {
 
 struct TcGeo {
     int L, d_k, d_v, r, C, n, NC;          // NC = chunks per sequence
+    int rm;                                // strict-mask group size (Problem::mask_group)
     uint32_t e_bytes, q_bytes, xi_bytes;   // per-chunk workspace record sizes
 };
 

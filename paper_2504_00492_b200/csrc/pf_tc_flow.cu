@@ -248,7 +248,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         // ---- epilogue 1: A -> X buffer (fp16) + fp32 diagonal blocks; P^T -> fp16 -------------------------
         {
             const int tokm = m / r;
-            const int row_lim = tokm * r;   // rows m' < row_lim belong to earlier tokens: tok(m') < tok(m)
+            const int row_lim = (m / g.rm) * g.rm;   // rows m' < row_lim: earlier tokens (sum form) / earlier rows (product form)
 #pragma unroll
             for (int c0 = 0; c0 < N; c0 += 32) {
                 uint32_t rr[32];

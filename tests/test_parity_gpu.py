@@ -179,7 +179,7 @@ TC_CASES = [
 ]
 
 
-def _run_with_status(w, impl):
+def _run_with_status(w, impl, mode="sum"):
     import paper_2504_00492_b200 as pf
     from paper_2504_00492_b200 import binding
     inp = pf_synth.make_inputs(w)
@@ -188,11 +188,12 @@ def _run_with_status(w, impl):
     assert need > 0
     ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
     off = (-ws.data_ptr()) % 256
-    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[off:off + need])
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[off:off + need],
+                                  mode=mode)
     torch.cuda.synchronize()
     status = int(ws[off:off + 4].view(torch.int32).item())
     assert status == 0, f"device-side wait {status} expired"
-    O_ref, Sf_ref = util.run_oracle(inp)
+    O_ref, Sf_ref = util.run_oracle(inp, mode=mode)
     return util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
 
 
@@ -287,3 +288,51 @@ def test_back_to_back_launches_without_synchronisation():
             first = (O.clone(), Sf.clone())
         else:
             assert torch.equal(O, first[0]) and torch.equal(Sf, first[1])
+
+
+# --- product form: the r factors of a token act one after another (mask strict in the flattened row index) -------
+
+@pytest.mark.parametrize("w", [w for w in SMALL if w.r > 1], ids=lambda w: w.name)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_product_mode_simt(w, dtype):
+    util.check_parity(w.with_(dtype=dtype), impl="simt", mode="product")
+
+
+@pytest.mark.parametrize("w", [w for w in TC_CASES if w.r > 1], ids=lambda w: w.name)
+@pytest.mark.parametrize("impl", ["tc_split", "tc_refflow"])
+def test_product_mode_two_launch_tensor_core_path(w, impl):
+    eo, es = _run_with_status(w, impl, mode="product")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+@pytest.mark.parametrize("w", [w for w in FUSED_CASES if w.r > 1], ids=lambda w: w.name)
+def test_product_mode_single_launch_path(w):
+    eo, es = _run_with_status(w, "tc", mode="product")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_product_mode_differs_from_sum_and_r1_does_not():
+    """The mode reaches the kernels (the two forms differ by far more than the tolerance for r = 2), and for
+    r = 1 the two are the same computation, bit for bit."""
+    import paper_2504_00492_b200 as pf
+    w = Workload("pm_r2", B=1, H=2, L=300, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=51)
+    d = pf_synth.make_inputs(w).to("cuda")
+    for impl in ("simt", "tc"):
+        Os, Ss = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl)
+        Op, Sp = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, mode="product")
+        assert util.max_rel(Op.cpu().numpy(), Os.cpu().numpy()) > 10 * util.TOL_BF16
+    w1 = w.with_(r=1)
+    d1 = pf_synth.make_inputs(w1).to("cuda")
+    for impl in ("simt", "tc"):
+        Os, Ss = pf.pf_deltanet_fwd_ex(d1.q, d1.k, d1.v, d1.beta, d1.S0, w1.chunk, impl=impl)
+        Op, Sp = pf.pf_deltanet_fwd_ex(d1.q, d1.k, d1.v, d1.beta, d1.S0, w1.chunk, impl=impl, mode="product")
+        assert torch.equal(Os, Op) and torch.equal(Ss, Sp)
+
+
+def test_unknown_mode_is_rejected():
+    import paper_2504_00492_b200 as pf
+    w = SMALL[1]
+    d = pf_synth.make_inputs(w).to("cuda")
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, mode=7)
+    assert e.value.status == -1
