@@ -42,6 +42,9 @@ def _load():
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int] * 6 + [ctypes.c_void_p] * 2 + [
                 ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+        lib.pf_oracle_deltanet_exact_fwd_f64.restype = ctypes.c_int
+        lib.pf_oracle_deltanet_exact_fwd_f64.argtypes = [ctypes.c_int] + [ctypes.c_void_p] * 5 + [ctypes.c_int] * 6 + [
+            ctypes.c_void_p] * 2 + [ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         _lib = lib
     return _lib
 
@@ -66,9 +69,12 @@ def _to_numpy(x):
     return np.asarray(x)
 
 
-def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: bool = False, mode: str = "sum"):
+def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: bool = False, mode: str = "sum",
+                 exact: bool = False):
     """Run the recurrence.  ``mode``: "sum" (all r factors of a token read the same old state: the paper's
-    rank-R form) or "product" (the factors act one after another: rank-1 delta rule r times per token).  Shapes: q [B,H,L,d_k], k [B,H,L,r,d_k], v [B,H,L,r,d_v], beta [B,H,L,r],
+    rank-R form) or "product" (the factors act one after another: rank-1 delta rule r times per token).
+    ``exact``: every rank-1 factor takes the exact step exp(-beta k k^T) instead of the Euler step I - beta k k^T
+    (r = 1, or the product form).  Shapes: q [B,H,L,d_k], k [B,H,L,r,d_k], v [B,H,L,r,d_v], beta [B,H,L,r],
     S0 [B,H,d_k,d_v] or None.  Inputs may be numpy or torch (bf16/fp16/fp32); they are widened
     exactly, the arithmetic is fp64.  Returns (O [B,H,L,d_v] float64, S_final [B,H,d_k,d_v] float64)
     and, if ``return_threads``, the number of host threads used."""
@@ -92,6 +98,9 @@ def deltanet_fwd(q, k, v, beta, S0=None, num_threads: int = 0, return_threads: b
     if mode not in ("sum", "product"):
         raise ValueError("mode must be 'sum' or 'product'")
     fn = _load().pf_oracle_deltanet_fwd_f64 if mode == "sum" else _load().pf_oracle_deltanet_product_fwd_f64
+    if exact:
+        base = _load().pf_oracle_deltanet_exact_fwd_f64
+        fn = lambda *a: base(1 if mode == "product" else 0, *a)
     rc = fn(
         qa.ctypes.data, ka.ctypes.data, va.ctypes.data, ba.ctypes.data,
         s0.ctypes.data if s0 is not None else None,

@@ -450,3 +450,51 @@ def test_chunk_form_with_flattened_mask_matches_product_recurrence(L, r, d_k, d_
     O_c, Sf_c, _ = pfm.chunked_forward(qd, kd, vd, bd, s0, chunk, product=True)
     np.testing.assert_allclose(O_c, O[0, 0], rtol=0, atol=1e-11)
     np.testing.assert_allclose(Sf_c, Sf[0, 0], rtol=0, atol=1e-11)
+
+
+# --- exact step of a rank-1 factor ("An alternative representation of the flow as product of exponentials") -----
+
+def test_exact_step_is_the_matrix_exponential():
+    # one token, v = 0: S_1 = S_0 exp(-beta k k^T), with the exponential from a library routine
+    import scipy.linalg
+    d_k, d_v = 6, 4
+    q, k, v, beta, S0 = make(90, L=1, r=1, d_k=d_k, d_v=d_v, beta_hi=3.0)
+    k = (k * 1.7).astype(np.float32)              # not unit norm: |k|^2 must enter the formula
+    v = np.zeros_like(v)
+    _, Sf = oracle.deltanet_fwd(q, k, v, beta, S0, exact=True)
+    kd, bd, s0 = f64(k[0, 0, 0, 0], beta[0, 0, 0, 0], S0[0, 0])
+    want = s0.T @ scipy.linalg.expm(-bd * np.outer(kd, kd))
+    np.testing.assert_allclose(Sf[0, 0], want.T, rtol=0, atol=TOL)
+
+
+@pytest.mark.parametrize("mode,r", [("sum", 1), ("product", 3)])
+def test_exact_step_is_the_limit_of_many_small_euler_steps(mode, r):
+    # a token split into N sub-steps of size beta / N (same k, v) is the Euler scheme on a finer grid: it converges,
+    # with error O(1/N), to the exact step -- for the input term as well as for the transition
+    L, d_k, d_v = 4, 5, 4
+    q, k, v, beta, S0 = make(91, L=L, r=r, d_k=d_k, d_v=d_v, beta_hi=1.5)
+    k = (k * 1.3).astype(np.float32)
+    O_x, Sf_x = oracle.deltanet_fwd(q, k, v, beta, S0, mode=mode, exact=True)
+    errs = []
+    for N in (200, 400):
+        # flatten to rank-1 factors, repeat each N times with beta / N: sub-steps act one after another
+        kf = np.repeat(k.reshape(1, 1, L * r, 1, d_k), N, axis=2)
+        vf = np.repeat(v.reshape(1, 1, L * r, 1, d_v), N, axis=2)
+        bf = np.repeat(beta.reshape(1, 1, L * r, 1).astype(np.float64) / N, N, axis=2).astype(np.float32)
+        qf = np.repeat(q, r * N, axis=2)
+        O_e, Sf_e = oracle.deltanet_fwd(qf, kf, vf, bf, S0)
+        errs.append(max(np.abs(O_e[:, :, r * N - 1::r * N] - O_x).max(), np.abs(Sf_e - Sf_x).max()))
+    assert errs[1] < 2e-2 and errs[1] < 0.6 * errs[0], errs      # first order in 1/N
+
+
+def test_exact_step_small_beta_limit_and_rank_restriction():
+    q, k, v, beta, S0 = make(92, L=6, r=1, d_k=5, d_v=4, beta_hi=1e-4)
+    O_e, Sf_e = oracle.deltanet_fwd(q, k, v, beta, S0)
+    O_x, Sf_x = oracle.deltanet_fwd(q, k, v, beta, S0, exact=True)
+    np.testing.assert_allclose(O_x, O_e, rtol=0, atol=1e-7)       # beta' = beta (1 - beta |k|^2 / 2 + ...)
+    q, k, v, beta, S0 = make(93, L=3, r=2, d_k=5, d_v=4)
+    with pytest.raises(RuntimeError):
+        oracle.deltanet_fwd(q, k, v, beta, S0, exact=True)        # sum form with r > 1: not rank 1
+    k0 = np.zeros_like(k[:, :, :, :1])
+    O_z, Sf_z = oracle.deltanet_fwd(q, k0, v[:, :, :, :1], beta[:, :, :, :1], S0, exact=True)
+    np.testing.assert_allclose(Sf_z, S0, rtol=0, atol=0)          # k = 0: nothing changes, no division by zero
