@@ -70,6 +70,18 @@ enum { PF_DTYPE_BF16 = 0, PF_DTYPE_F32 = 1 };
  *                     other formula is unchanged.  Every factor is a contraction for beta in [0, 2]. */
 enum { PF_MODE_SUM = 0, PF_MODE_PRODUCT = 1 };
 
+/* How one rank-1 factor advances the state (pf_params.step).
+ *   PF_STEP_EULER : S <- S (I - beta k k^T) + beta v k^T, the discretisation the paper's chunk algorithms use
+ *                   (Eq. (discretization), Section 3.1).  Default.
+ *   PF_STEP_EXACT : the exact solution of the same linear equation over the step, from the subsection "An
+ *                   alternative representation of the flow as product of exponentials":
+ *                       exp(-beta k k^T) = I - beta' k k^T,   beta' = (1 - e^{-beta |k|^2}) / |k|^2,
+ *                   and the input term takes the same beta'.  It is the delta rule with beta' in place of beta,
+ *                   computed by one extra kernel before the others (fp32, one warp per factor; beta' = beta
+ *                   where k = 0).  Defined for rank-1 factors: r = 1, or PF_MODE_PRODUCT with any r; the sum
+ *                   form with r > 1 returns PF_ERR_UNSUPPORTED.  beta' < 1/|k|^2, so every factor contracts. */
+enum { PF_STEP_EULER = 0, PF_STEP_EXACT = 1 };
+
 /* Which kernels evaluate the chunk form.
  *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
@@ -147,11 +159,13 @@ typedef struct pf_params {
     size_t workspace_bytes;
     void* stream;
     int mode;                 /* PF_MODE_SUM (0) or PF_MODE_PRODUCT; anything else: PF_ERR_INVALID */
+    int step;                 /* PF_STEP_EULER (0) or PF_STEP_EXACT; anything else: PF_ERR_INVALID */
 } pf_params;
 
 /* Same operation with explicit options.  The workspace holds per-chunk intermediates (T', W, Uh, P
- * of Theorem 3.2 in the forms the selected kernels exchange); its content after the call is
- * unspecified.  Same passages as pf_deltanet_fwd. */
+ * of Theorem 3.2 in the forms the selected kernels exchange) and, at its end, the fp32 step sizes of
+ * PF_STEP_EXACT; its content after the call is unspecified.  Same passages as pf_deltanet_fwd, plus those
+ * named at PF_MODE_* and PF_STEP_*. */
 int pf_deltanet_fwd_ex(const pf_params* p);
 
 /* Bytes of scratch pf_deltanet_fwd_ex needs for this problem with this in_dtype/impl (0 on an

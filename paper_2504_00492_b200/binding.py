@@ -21,6 +21,8 @@ PF_IMPL_TC_REFFLOW = 3
 PF_IMPL_TC_SPLIT = 4
 PF_MODE_SUM, PF_MODE_PRODUCT = 0, 1
 MODE_BY_NAME = {"sum": PF_MODE_SUM, "product": PF_MODE_PRODUCT}
+PF_STEP_EULER, PF_STEP_EXACT = 0, 1
+STEP_BY_NAME = {"euler": PF_STEP_EULER, "exact": PF_STEP_EXACT}
 IMPL_BY_NAME = {"auto": PF_IMPL_AUTO, "simt": PF_IMPL_SIMT, "tc": PF_IMPL_TC, "tc_refflow": PF_IMPL_TC_REFFLOW,
                 "tc_split": PF_IMPL_TC_SPLIT}
 
@@ -44,6 +46,7 @@ class PfParams(ctypes.Structure):
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p),
         ("mode", ctypes.c_int),
+        ("step", ctypes.c_int),
     ]
 
 
@@ -185,10 +188,11 @@ def pf_static_scratch_bytes() -> int:
 
 
 def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Optional[torch.Tensor] = None,
-                       O=None, S_final=None, stream=None, want_state: bool = True, mode="sum"):
+                       O=None, S_final=None, stream=None, want_state: bool = True, mode="sum", step="euler"):
     """Same operation with an explicit implementation and (optionally) a caller-owned workspace
     (a uint8 CUDA tensor of at least pf_workspace_bytes(...) bytes).  mode: "sum" (the r factors of a token
-    read the same previous state) or "product" (they act one after another)."""
+    read the same previous state) or "product" (they act one after another).  step: "euler" (the paper's
+    discretisation) or "exact" (each rank-1 factor takes exp(-beta k k^T); r = 1 or the product form)."""
     dtype = q.dtype
     if dtype not in (torch.bfloat16, torch.float32):
         raise TypeError("q/k/v/beta must be bf16 or fp32")
@@ -204,6 +208,7 @@ def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Op
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.stream = _stream(stream)
     p.mode = MODE_BY_NAME[mode] if isinstance(mode, str) else int(mode)
+    p.step = STEP_BY_NAME[step] if isinstance(step, str) else int(step)
     with torch.cuda.device(q.device):
         st = lib().pf_deltanet_fwd_ex(ctypes.byref(p))
     if st != 0:

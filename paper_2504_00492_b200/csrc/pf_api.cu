@@ -76,11 +76,36 @@ int select_impl(const Problem& p, int impl) {
     }
 }
 
-size_t workspace_need(const Problem& p, int impl) {
+// what the kernels of `impl` carve up (the fp32 step sizes of PF_STEP_EXACT follow it)
+size_t kernel_workspace_need(const Problem& p, int impl) {
     if (impl == PF_IMPL_TC) return fused_supported(p) ? fused_workspace_bytes(p) : tc_workspace_bytes(p);
     if (impl == PF_IMPL_TC_SPLIT) return tc_workspace_bytes(p);
     if (impl == PF_IMPL_TC_REFFLOW) return tc_refflow_workspace_bytes(p);
     return simt_workspace_bytes(p);
+}
+size_t workspace_need(const Problem& p, int impl) {
+    return align_up(kernel_workspace_need(p, impl), 256) + beta32_bytes(p);
+}
+
+// PF_STEP_EXACT: beta'[m] = (1 - e^{-beta_m |k_m|^2}) / |k_m|^2 for every factor m (a row of k); beta_m where k_m = 0.
+// One warp per row.
+template <class Tin>
+__global__ void __launch_bounds__(256) exact_steps_kernel(const Tin* __restrict__ k, const Tin* __restrict__ beta,
+                                                          float* __restrict__ out, long long rows, int d_k) {
+    const long long m = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (m >= rows) return;
+    const int lane = threadIdx.x & 31;
+    float s = 0.f;
+    for (int i = lane; i < d_k; i += 32) {
+        const float x = (float)k[m * d_k + i];
+        s = fmaf(x, x, s);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+        const float b = (float)beta[m];
+        out[m] = s > 0.f ? -expm1f(-b * s) / s : b;
+    }
 }
 
 bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
@@ -94,6 +119,8 @@ int forward(const pf_params* a) {
     int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
     if (st != PF_OK) return st;
     if (a->mode != PF_MODE_SUM && a->mode != PF_MODE_PRODUCT) return PF_ERR_INVALID;
+    if (a->step != PF_STEP_EULER && a->step != PF_STEP_EXACT) return PF_ERR_INVALID;
+    if (a->step == PF_STEP_EXACT && a->mode == PF_MODE_SUM && a->r != 1) return PF_ERR_UNSUPPORTED;   // rank-1 factors only
     Problem p = as_problem(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk, a->in_dtype);
     p.mode = a->mode;
     const int impl = select_impl(p, a->impl);
@@ -130,6 +157,25 @@ int forward(const pf_params* a) {
     }
     g_launch_accum = 0;
     g_prof_n = 0;
+    const long long rows = (long long)p.B * p.H * p.L * p.r;
+    if (a->step == PF_STEP_EXACT && rows > 0) {
+        float* b32 = (float*)((uint8_t*)ws + align_up(kernel_workspace_need(p, impl), 256));
+        const unsigned grid = (unsigned)((rows + 7) / 8);
+        prof_begin("exact_steps", p.stream);
+        if (p.in_dtype == PF_DTYPE_F32)
+            exact_steps_kernel<float><<<grid, 256, 0, p.stream>>>((const float*)p.k, (const float*)p.beta, b32, rows, p.d_k);
+        else
+            exact_steps_kernel<__nv_bfloat16><<<grid, 256, 0, p.stream>>>((const __nv_bfloat16*)p.k,
+                                                                          (const __nv_bfloat16*)p.beta, b32, rows, p.d_k);
+        prof_end(p.stream);
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) {
+            if (own) cudaFreeAsync(ws, p.stream);
+            return record_cuda_error(e, "exact_steps_kernel");
+        }
+        p.beta32 = b32;
+    }
     if (impl == PF_IMPL_TC) st = fused_supported(p) ? fused_forward(p, ws) : tc_forward(p, ws);
     else if (impl == PF_IMPL_TC_SPLIT) st = tc_forward(p, ws);
     else if (impl == PF_IMPL_TC_REFFLOW) st = tc_forward_refflow(p, ws);

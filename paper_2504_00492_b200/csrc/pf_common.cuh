@@ -23,6 +23,7 @@ struct Problem {
     float* S_final;
     int in_dtype;
     int mode;           // PF_MODE_SUM (0) or PF_MODE_PRODUCT
+    const float* beta32;    // null, or fp32 step sizes [B,H,L,r] (device) that the kernels use in place of beta
     cudaStream_t stream;
 
     __host__ __device__ int n() const { return chunk * r; }            // rows per chunk
@@ -49,6 +50,8 @@ void prof_begin(const char* name, cudaStream_t stream);
 void prof_end(cudaStream_t stream);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// room at the end of every workspace for the fp32 step sizes of PF_STEP_EXACT
+inline size_t beta32_bytes(const Problem& p) { return align_up((size_t)p.B * p.H * p.L * p.r * 4, 256); }
 
 // fp32 SIMT path (pf_simt.cu)
 size_t simt_workspace_bytes(const Problem& p);

@@ -66,6 +66,7 @@ constexpr uint32_t SLOT_BYTES = SLOT_XI + DK * DV * 2;  // 81920
 struct FusedGeo {
     int L, r, C, NC, nseq, R;
     int rm;             // strict-mask group size (Problem::mask_group)
+    const float* b32;   // null, or fp32 step sizes used in place of beta (Problem::beta32)
     int n_scan, n_flow;
     int items;          // nseq * NC
 };
@@ -325,7 +326,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             int seq, c;
             item(0, seq, c);
             const int nv = min(C, g.L - c * C) * r;
-            if (m < nv) beta_next = __bfloat162float(beta[((long long)seq * g.L + (long long)c * C) * r + m]);
+            if (m < nv) {
+                    const long long bi = ((long long)seq * g.L + (long long)c * C) * r + m;
+                    beta_next = g.b32 ? g.b32[bi] : __bfloat162float(beta[bi]);
+                }
         }
 #pragma unroll 1
         for (int k = 0; k < nk; ++k) {
@@ -339,7 +343,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 int seq, c;
                 item(k + 1, seq, c);
                 const int nv = min(C, g.L - c * C) * r;
-                if (m < nv) beta_next = __bfloat162float(beta[((long long)seq * g.L + (long long)c * C) * r + m]);
+                if (m < nv) {
+                    const long long bi = ((long long)seq * g.L + (long long)c * C) * r + m;
+                    beta_next = g.b32 ? g.b32[bi] : __bfloat162float(beta[bi]);
+                }
             }
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
@@ -1171,7 +1178,7 @@ int fused_forward(const Problem& p, void* workspace) {
     ws.ring = base + cv.ring;
     PF_CUDA_TRY(cudaMemsetAsync(base, 0, cv.flag_bytes, p.stream));
     FusedGeo g{};
-    g.L = p.L; g.r = p.r; g.C = p.chunk; g.NC = NC; g.nseq = nseq; g.R = ring_depth(p); g.rm = p.mask_group();
+    g.L = p.L; g.r = p.r; g.C = p.chunk; g.NC = NC; g.nseq = nseq; g.R = ring_depth(p); g.rm = p.mask_group(); g.b32 = p.beta32;
     g.items = nseq * NC;
     const int sms = sm_count();
     g.n_scan = nseq;

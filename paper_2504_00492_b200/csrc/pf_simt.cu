@@ -25,6 +25,7 @@ template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloa
 struct Geo {
     int L, d_k, d_v, r, C, n, NC;   // NC = chunks per sequence
     int rm;                         // strict-mask group size (Problem::mask_group)
+    const float* b32;               // null, or fp32 step sizes used in place of beta (Problem::beta32)
 };
 
 // Workspace (fp32), G = total chunks:  T [G][n][n]  W [G][n][d_k]  U [G][n][d_v]  P [G][C][n]
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(256) simt_gram(const Tin* __restrict__ q, cons
             for (int i = 0; i < 4; ++i) {
                 const int m = m0 + ty * 4 + i;
                 if (m >= n) continue;
-                const float bm = (m < nv) ? ldf(bc + m) : 0.f;
+                const float bm = (m < nv) ? (g.b32 ? g.b32[(seq * g.L + t0) * (long long)r + m] : ldf(bc + m)) : 0.f;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int mp = n0 + tx * 4 + j;
@@ -175,7 +176,7 @@ __global__ void simt_solve(const Tin* __restrict__ beta, Geo g, Ws ws) {
     const Tin* bc = beta + (seq * g.L + t0) * (long long)r;
     float* Tg = ws.T + gc * (long long)n * n;
     const int c = threadIdx.x;
-    const float bcol = (c < nv) ? ldf(bc + c) : 0.f;
+    const float bcol = (c < nv) ? (g.b32 ? g.b32[(seq * g.L + t0) * (long long)r + c] : ldf(bc + c)) : 0.f;
     const int wstart = (c / 32) * 32;                // first column of this warp: warp-uniform loop start
 
     for (int m0 = 0; m0 < n; m0 += RB) {
@@ -366,7 +367,7 @@ Ws carve(const Problem& p, void* workspace) {
 
 template <class Tin>
 int run(const Problem& p, void* workspace, bool prepare_only) {
-    Geo g{p.L, p.d_k, p.d_v, p.r, p.chunk, p.n(), p.chunks_per_seq(), p.mask_group()};
+    Geo g{p.L, p.d_k, p.d_v, p.r, p.chunk, p.n(), p.chunks_per_seq(), p.mask_group(), p.beta32};
     const long long G = p.total_chunks();
     const long long nseq = (long long)p.B * p.H;
     const Tin* q = (const Tin*)p.q;

@@ -277,7 +277,7 @@ int pick_dvs(const Problem& p) {
 
 TcGeo tc_geo(const Problem& p) {
     TcGeo g{};
-    g.L = p.L; g.d_k = p.d_k; g.d_v = p.d_v; g.r = p.r; g.C = p.chunk; g.n = p.n(); g.NC = p.chunks_per_seq(); g.rm = p.mask_group();
+    g.L = p.L; g.d_k = p.d_k; g.d_v = p.d_v; g.r = p.r; g.C = p.chunk; g.n = p.n(); g.NC = p.chunks_per_seq(); g.rm = p.mask_group(); g.b32 = p.beta32;
     g.e_bytes = (uint32_t)p.d_k * p.d_k * 2;
     g.q_bytes = (uint32_t)p.d_k * 128;
     g.xi_bytes = (uint32_t)p.d_k * p.d_v * 2;

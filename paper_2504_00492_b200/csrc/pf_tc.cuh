@@ -8,6 +8,7 @@ namespace pf {
 struct TcGeo {
     int L, d_k, d_v, r, C, n, NC;          // NC = chunks per sequence
     int rm;                                // strict-mask group size (Problem::mask_group)
+    const float* b32;                      // null, or fp32 step sizes used in place of beta (Problem::beta32)
     uint32_t e_bytes, q_bytes, xi_bytes;   // per-chunk workspace record sizes
 };
 

@@ -207,7 +207,10 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         const int m = tid;
         float beta_m = 0.f;
-        if (m < nv) beta_m = __bfloat162float(beta[(seq * g.L + t0) * (long long)r + m]);
+        if (m < nv) {
+            const long long bi = (seq * g.L + t0) * (long long)r + m;
+            beta_m = g.b32 ? g.b32[bi] : __bfloat162float(beta[bi]);
+        }
         if (m < N) sBeta[m] = __float2half_rn(beta_m);
         ok = mbar_wait(&tma_bar, tma_phase, err, 21);
         tma_phase ^= 1;

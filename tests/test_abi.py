@@ -53,11 +53,12 @@ def test_shape_checks_need_no_gpu(kw, code):
 
 
 def test_simt_workspace_arithmetic():
-    # T [G][n][n] + W [G][n][d_k] + U [G][n][d_v] + P [G][C][n], fp32, each 256-byte aligned
+    # T [G][n][n] + W [G][n][d_k] + U [G][n][d_v] + P [G][C][n], fp32, each 256-byte aligned, then room for the fp32
+    # step sizes of PF_STEP_EXACT [B,H,L,r]
     B, H, L, d_k, d_v, r, C = 2, 3, 100, 64, 128, 3, 32
     G, n = B * H * ((L + C - 1) // C), C * r
     al = lambda x: (x + 255) // 256 * 256
-    want = al(G * n * n * 4) + al(G * n * d_k * 4) + al(G * n * d_v * 4) + al(G * C * n * 4) + 256
+    want = al(G * n * n * 4) + al(G * n * d_k * 4) + al(G * n * d_v * 4) + al(G * C * n * 4) + 256 + al(B * H * L * r * 4)
     assert pf.pf_workspace_bytes(B, H, L, d_k, d_v, r, C, binding.PF_DTYPE_F32, "simt") == want
     assert pf.pf_select_impl(B, H, L, d_k, d_v, r, C, binding.PF_DTYPE_F32, "auto") == binding.PF_IMPL_SIMT
     assert pf.pf_select_impl(B, H, L, d_k, d_v, r, C, binding.PF_DTYPE_F32, "tc") == -2

@@ -179,7 +179,7 @@ TC_CASES = [
 ]
 
 
-def _run_with_status(w, impl, mode="sum"):
+def _run_with_status(w, impl, mode="sum", step="euler"):
     import paper_2504_00492_b200 as pf
     from paper_2504_00492_b200 import binding
     inp = pf_synth.make_inputs(w)
@@ -189,11 +189,11 @@ def _run_with_status(w, impl, mode="sum"):
     ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
     off = (-ws.data_ptr()) % 256
     O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[off:off + need],
-                                  mode=mode)
+                                  mode=mode, step=step)
     torch.cuda.synchronize()
     status = int(ws[off:off + 4].view(torch.int32).item())
     assert status == 0, f"device-side wait {status} expired"
-    O_ref, Sf_ref = util.run_oracle(inp, mode=mode)
+    O_ref, Sf_ref = util.run_oracle(inp, mode=mode, step=step)
     return util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
 
 
@@ -335,4 +335,46 @@ def test_unknown_mode_is_rejected():
     d = pf_synth.make_inputs(w).to("cuda")
     with pytest.raises(pf.PfError) as e:
         pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, mode=7)
+    assert e.value.status == -1
+
+
+# --- exact step of a rank-1 factor: exp(-beta k k^T) instead of I - beta k k^T ---------------------------------------
+
+EXACT_CASES = [   # (workload, impl, mode): r = 1 in the sum form, any r in the product form; beta up to 2
+    (SMALL[0].with_(dtype="f32"), "simt", "sum"),
+    (SMALL[0], "simt", "sum"),
+    (SMALL[3], "simt", "product"),
+    (SMALL[2].with_(dtype="f32"), "simt", "product"),
+    (TC_CASES[2], "tc_split", "sum"),
+    (TC_CASES[3], "tc_split", "product"),
+    (TC_CASES[4], "tc_refflow", "product"),
+    (FUSED_CASES[2], "tc", "sum"),
+    (FUSED_CASES[0], "tc", "product"),
+    (FUSED_CASES[1], "tc", "product"),
+]
+
+
+@pytest.mark.parametrize("w,impl,mode", EXACT_CASES, ids=lambda x: getattr(x, "name", x))
+def test_exact_step(w, impl, mode):
+    if impl == "simt":
+        util.check_parity(w, impl=impl, mode=mode, step="exact")
+    else:
+        eo, es = _run_with_status(w, impl, mode=mode, step="exact")
+        assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_exact_step_changes_the_result_and_needs_rank_one_factors():
+    import paper_2504_00492_b200 as pf
+    w = TC_CASES[2]                                    # r = 1
+    d = pf_synth.make_inputs(w).to("cuda")
+    O1, _ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    O2, _ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, step="exact")
+    assert util.max_rel(O2.cpu().numpy(), O1.cpu().numpy()) > 10 * util.TOL_BF16
+    w2 = TC_CASES[0]                                   # r = 2, sum form: not rank 1
+    d2 = pf_synth.make_inputs(w2).to("cuda")
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk, step="exact")
+    assert e.value.status == -2
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk, step=5)
     assert e.value.status == -1

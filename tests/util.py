@@ -23,24 +23,25 @@ def max_rel(x, ref) -> float:
     return float(np.abs(x - ref).max() / den)
 
 
-def run_gpu(w: pf_synth.Workload, inp: pf_synth.Inputs, impl="auto", chunk=None, workspace=None, mode="sum"):
+def run_gpu(w: pf_synth.Workload, inp: pf_synth.Inputs, impl="auto", chunk=None, workspace=None, mode="sum",
+            step="euler"):
     import paper_2504_00492_b200 as pf
     d = inp.to("cuda")
     O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, chunk or w.chunk, impl=impl, workspace=workspace,
-                                  mode=mode)
+                                  mode=mode, step=step)
     torch.cuda.synchronize()
     return O.cpu().numpy(), Sf.cpu().numpy()
 
 
-def run_oracle(inp: pf_synth.Inputs, mode="sum"):
-    return oracle.deltanet_fwd(inp.q, inp.k, inp.v, inp.beta, inp.S0, mode=mode)
+def run_oracle(inp: pf_synth.Inputs, mode="sum", step="euler"):
+    return oracle.deltanet_fwd(inp.q, inp.k, inp.v, inp.beta, inp.S0, mode=mode, exact=(step == "exact"))
 
 
-def check_parity(w: pf_synth.Workload, impl="auto", tol=None, inp=None, mode="sum"):
+def check_parity(w: pf_synth.Workload, impl="auto", tol=None, inp=None, mode="sum", step="euler"):
     inp = inp or pf_synth.make_inputs(w)
     tol = tol if tol is not None else (TOL_F32 if w.dtype == "f32" else TOL_BF16)
-    O, Sf = run_gpu(w, inp, impl=impl, mode=mode)
-    O_ref, Sf_ref = run_oracle(inp, mode=mode)
+    O, Sf = run_gpu(w, inp, impl=impl, mode=mode, step=step)
+    O_ref, Sf_ref = run_oracle(inp, mode=mode, step=step)
     assert np.isfinite(O).all() and np.isfinite(Sf).all()
     eo, es = max_rel(O, O_ref), max_rel(Sf, Sf_ref)
     assert eo <= tol, f"{w.name}: O error {eo:.3e} > {tol}"
