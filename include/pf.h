@@ -176,10 +176,15 @@ size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chun
 /* Which PF_IMPL_* pf_deltanet_fwd_ex would run for this problem (negative pf_status if none). */
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
 
-/* Tuning knobs (process-wide, not thread-safe; results do not depend on them).  Returns PF_OK,
+/* Knobs (process-wide, not thread-safe; results agree within rounding whatever their values).  Returns PF_OK,
  * PF_ERR_UNSUPPORTED for an unknown name, PF_ERR_INVALID for a value out of range.
  *   "ring_depth" (3..64, default 8): slots per sequence of the L2-resident ring through which the
- *       single-launch tensor-core path hands each chunk's flow to the state scan. */
+ *       single-launch tensor-core path hands each chunk's flow to the state scan.
+ *   "wu_builder" (0 or 1, default 0): how the fp32 SIMT kernels obtain W and Uh of a chunk.  0: the triangular
+ *       inverse T' of Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
+ *       "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one kernel; it
+ *       needs more workspace (pf_workspace_bytes follows the current value).  The tensor-core kernels do not
+ *       use it, except PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels. */
 int pf_set_option(const char* name, int value);
 
 /* Number of kernels the last successful call on this host thread enqueued. */

@@ -57,10 +57,13 @@ int check_shape(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
     return PF_OK;
 }
 
+int g_wu_builder = 0;     // option "wu_builder"
+
 Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype) {
     Problem p{};
     p.B = B; p.H = H; p.L = L; p.d_k = d_k; p.d_v = d_v; p.r = r; p.chunk = chunk;
     p.in_dtype = in_dtype;
+    p.wu_builder = g_wu_builder;
     return p;
 }
 
@@ -239,6 +242,11 @@ int pf_last_launch_count(void) { return pf::g_launches; }
 
 int pf_set_option(const char* name, int value) {
     if (!name) return PF_ERR_INVALID;
+    if (strcmp(name, "wu_builder") == 0) {
+        if (value != 0 && value != 1) return PF_ERR_INVALID;
+        pf::g_wu_builder = value;
+        return PF_OK;
+    }
     return pf::fused_set_option(name, value);
 }
 

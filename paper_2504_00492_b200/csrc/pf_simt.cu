@@ -8,6 +8,10 @@
 //   simt_scan   per (b, h, d_v slice), serial over chunks:
 //               U' = Uh - W S^T,  O = Q S^T + P U',  S <- S + U'^T K
 //
+// With option "wu_builder" = 1, simt_solve and simt_wu are replaced by simt_sigdelta, which obtains the same W and Uh
+// from the two-index system of Theorem 3.3 (the "signature kernel inspired algorithm"), swept along its
+// antidiagonals.
+//
 // Rows of a chunk are m = t*r + j (token t, factor j), n = chunk*r.  Rows past the end of the
 // sequence behave as beta = 0, k = 0, which leaves the state untouched; their outputs are not stored.
 #include "pf_common.cuh"
@@ -34,6 +38,7 @@ struct Ws {
     float* W;
     float* U;
     float* P;
+    double* D;      // wu_builder 1 only: [G][3][cells_max][r][d_k + d_v], three antidiagonals of the two-index system
 };
 
 // ------------------------------------------------------------------------------------------
@@ -350,6 +355,101 @@ __global__ void __launch_bounds__(256) simt_scan(const Tin* __restrict__ q, cons
         }
 }
 
+// ------------------------------------------------------------------------------------------
+// simt_sigdelta: one CTA per chunk.  Theorem 3.3: the solution W_{t_k} of
+//     W_{t_k} = A_{t_k} + sum_{m<k} W_{t_m} B_{t_m}^T A_{t_k}
+// is the diagonal W(t_k, t_k) of the system
+//     W(t_0, t_k) = A_{t_k},
+//     W(t_{k+1}, t_{k+1}) = W(t_k, t_{k+1}) + W(t_k, t_k) B_{t_k}^T A_{t_{k+1}},
+//     W(t_{m+1}, t_{k+1}) = W(t_m, t_{k+1}) + W(t_{m+1}, t_k) - W(t_m, t_k) + W(t_m, t_m) B_{t_m}^T (A_{t_{k+1}} - A_{t_k})   (m < k).
+// A cell (m, k), m <= k, holds the R rows of token k (d_k values of W, then d_v values of the same system driven by
+// V, which gives Uh).  Cells with the same m + k do not depend on each other: the grid is swept antidiagonal by
+// antidiagonal (2C - 1 steps), all cells of one antidiagonal at once, with the two previous antidiagonals kept in
+// global memory (L2).  In the row notation used here  A_{t_k} -> rows beta_m k_m,  and the R x R coefficients
+// B_{t_m}^T A_{t_k} are, up to sign, the entries A[(k,j)][(m,i)] = beta_(k,j) k_(k,j).k_(m,i) that simt_gram left in T.
+// Product form: the same system with every row a token of its own (C*r tokens, R = 1).
+// The cells are kept in fp64: each update adds two neighbours and subtracts a third, all of the size of the result,
+// 2C - 1 times in a row, and in fp32 that alone costs 2e-5 of max|O| at 256 rows, more than the fp32 entry point is
+// allowed in total.  Inputs, coefficients and the finished rows of W and Uh stay fp32.
+// ------------------------------------------------------------------------------------------
+template <class Tin>
+__global__ void __launch_bounds__(256) simt_sigdelta(const Tin* __restrict__ k, const Tin* __restrict__ v,
+                                                     const Tin* __restrict__ beta, Geo g, Ws ws, int cells_max) {
+    const long long gc = blockIdx.x;
+    const long long seq = gc / g.NC;
+    const int ci = (int)(gc % g.NC);
+    const int t0 = ci * g.C;
+    const int n = g.n, d_k = g.d_k, d_v = g.d_v, DT = g.d_k + g.d_v;
+    const int nv = min(g.C, g.L - t0) * g.r;
+    const int R = g.rm;                 // rows per token of the system: r (sum form) or 1 (product form)
+    const int CT = n / R;               // tokens of the system
+    const Tin* Kc = k + ((seq * g.L + t0) * g.r) * (long long)d_k;
+    const Tin* Vc = v + ((seq * g.L + t0) * g.r) * (long long)d_v;
+    const Tin* bc = beta + (seq * g.L + t0) * (long long)g.r;
+    const float* Tg = ws.T + gc * (long long)n * n;
+    float* Wg = ws.W + gc * (long long)n * d_k;
+    float* Ug = ws.U + gc * (long long)n * d_v;
+    double* Dg = ws.D + gc * 3ll * cells_max * R * DT;
+    const long long dstride = (long long)cells_max * R * DT;
+    auto m_lo = [&](int s) { return max(0, s - (CT - 1)); };
+
+    for (int s = 0; s <= 2 * (CT - 1); ++s) {
+        const int lo = m_lo(s), hi = s >> 1;
+        const int total = (hi - lo + 1) * R * DT;
+        double* Ds = Dg + (s % 3) * dstride;
+        const double* D1 = Dg + ((s + 2) % 3) * dstride;    // antidiagonal s - 1
+        const double* D2 = Dg + ((s + 1) % 3) * dstride;    // antidiagonal s - 2
+        const int lo1 = m_lo(s - 1), lo2 = m_lo(s - 2);
+        for (int e = threadIdx.x; e < total; e += 256) {
+            const int x = e % DT;
+            const int j = (e / DT) % R;
+            const int m = lo + e / (DT * R);
+            const int kk = s - m;
+            const int row = kk * R + j;
+            double val;
+            if (m == 0) {
+                float b = 0.f, a = 0.f;
+                if (row < nv) {
+                    b = g.b32 ? g.b32[(seq * g.L + t0) * (long long)g.r + row] : ldf(bc + row);
+                    a = (x < d_k) ? ldf(Kc + (long long)row * d_k + x) : ldf(Vc + (long long)row * d_v + (x - d_k));
+                }
+                val = (double)(b * a);                                          // W(t_0, t_k) = A_{t_k}
+            } else {
+                const float* fin = (x < d_k) ? (Wg + (long long)(m - 1) * R * d_k + x) : (Ug + (long long)(m - 1) * R * d_v + (x - d_k));
+                const int fstride = (x < d_k) ? d_k : d_v;
+                const long long c1 = ((long long)(m - 1 - lo1) * R + j) * DT + x;            // (m-1, k)   on s - 1
+                double acc = 0.0;
+                if (m == kk) {
+                    val = D1[c1];
+                    for (int i = 0; i < R; ++i)
+                        acc += (double)(fin[(long long)i * fstride] * Tg[(long long)row * n + (m - 1) * R + i]);
+                } else {
+                    const long long c2 = ((long long)(m - lo1) * R + j) * DT + x;            // (m, k-1)   on s - 1
+                    const long long c3 = ((long long)(m - 1 - lo2) * R + j) * DT + x;        // (m-1, k-1) on s - 2
+                    val = D1[c1] + D1[c2] - D2[c3];
+                    for (int i = 0; i < R; ++i)
+                        acc += (double)fin[(long long)i * fstride] *
+                               ((double)Tg[(long long)row * n + (m - 1) * R + i] - (double)Tg[(long long)(row - R) * n + (m - 1) * R + i]);
+                }
+                val -= acc;
+            }
+            Ds[((long long)(m - lo) * R + j) * DT + x] = val;
+            if (m == kk) {                                                      // diagonal cell: W_{t_k} itself
+                if (x < d_k) Wg[(long long)row * d_k + x] = (float)val;
+                else Ug[(long long)row * d_v + (x - d_k)] = (float)val;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// cells on the longest antidiagonal of the two-index system
+int sigdelta_cells_max(const Problem& p) { return (p.n() / p.mask_group()) / 2 + 1; }
+size_t sigdelta_bytes(const Problem& p) {
+    if (!p.wu_builder) return 0;
+    return align_up((size_t)p.total_chunks() * 3 * sigdelta_cells_max(p) * p.mask_group() * (p.d_k + p.d_v) * sizeof(double), 256);
+}
+
 Ws carve(const Problem& p, void* workspace) {
     const size_t G = (size_t)p.total_chunks();
     const size_t n = p.n();
@@ -362,6 +462,8 @@ Ws carve(const Problem& p, void* workspace) {
     ws.U = (float*)base;
     base += align_up(G * n * p.d_v * sizeof(float), 256);
     ws.P = (float*)base;
+    base += align_up(G * (size_t)p.chunk * n * sizeof(float), 256);
+    ws.D = p.wu_builder ? (double*)base : nullptr;
     return ws;
 }
 
@@ -385,13 +487,20 @@ int run(const Problem& p, void* workspace, bool prepare_only) {
         prof_begin("simt_gram", p.stream);
         simt_gram<Tin><<<(unsigned)G, 256, 0, p.stream>>>(q, k, beta, g, ws);
         prof_end(p.stream);
-        prof_begin("simt_solve", p.stream);
-        simt_solve<Tin><<<(unsigned)G, g.n, solve_smem, p.stream>>>(beta, g, ws);
-        prof_end(p.stream);
-        prof_begin("simt_wu", p.stream);
-        simt_wu<Tin><<<(unsigned)G, 256, 0, p.stream>>>(k, v, g, ws);
-        prof_end(p.stream);
-        launches += 3;
+        if (p.wu_builder) {
+            prof_begin("simt_sigdelta", p.stream);
+            simt_sigdelta<Tin><<<(unsigned)G, 256, 0, p.stream>>>(k, v, beta, g, ws, sigdelta_cells_max(p));
+            prof_end(p.stream);
+            launches += 2;
+        } else {
+            prof_begin("simt_solve", p.stream);
+            simt_solve<Tin><<<(unsigned)G, g.n, solve_smem, p.stream>>>(beta, g, ws);
+            prof_end(p.stream);
+            prof_begin("simt_wu", p.stream);
+            simt_wu<Tin><<<(unsigned)G, 256, 0, p.stream>>>(k, v, g, ws);
+            prof_end(p.stream);
+            launches += 3;
+        }
     }
     if (prepare_only) {
         PF_CUDA_TRY(cudaGetLastError());
@@ -414,7 +523,8 @@ size_t simt_workspace_bytes(const Problem& p) {
     const size_t G = (size_t)p.total_chunks();
     const size_t n = p.n();
     return align_up(G * n * n * sizeof(float), 256) + align_up(G * n * p.d_k * sizeof(float), 256) +
-           align_up(G * n * p.d_v * sizeof(float), 256) + align_up(G * (size_t)p.chunk * n * sizeof(float), 256) + 256;
+           align_up(G * n * p.d_v * sizeof(float), 256) + align_up(G * (size_t)p.chunk * n * sizeof(float), 256) +
+           sigdelta_bytes(p) + 256;
 }
 
 int simt_forward(const Problem& p, void* workspace) {

@@ -378,3 +378,49 @@ def test_exact_step_changes_the_result_and_needs_rank_one_factors():
     with pytest.raises(pf.PfError) as e:
         pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk, step=5)
     assert e.value.status == -1
+
+
+# --- W and Uh from the two-index system of Theorem 3.3 (option "wu_builder" = 1) instead of the triangular inverse ----
+
+@pytest.fixture
+def wavefront_builder():
+    import paper_2504_00492_b200 as pf
+    pf.pf_set_option("wu_builder", 1)
+    yield
+    pf.pf_set_option("wu_builder", 0)
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_theorem_3_3_builder_simt(wavefront_builder, w, dtype):
+    util.check_parity(w.with_(dtype=dtype), impl="simt")
+
+
+@pytest.mark.parametrize("w", [SMALL[1], SMALL[3]], ids=lambda w: w.name)
+def test_theorem_3_3_builder_product_form_and_exact_step(wavefront_builder, w):
+    util.check_parity(w.with_(dtype="f32"), impl="simt", mode="product")
+    util.check_parity(w, impl="simt", mode="product", step="exact")
+
+
+def test_theorem_3_3_builder_feeds_the_tensor_core_scan(wavefront_builder):
+    eo, es = _run_with_status(TC_CASES[0], "tc_refflow")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_the_two_builders_agree_closely_and_the_option_is_checked():
+    import paper_2504_00492_b200 as pf
+    w = SMALL[3].with_(dtype="f32")
+    d = pf_synth.make_inputs(w).to("cuda")
+    O0, S0_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt")
+    need0 = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt")
+    pf.pf_set_option("wu_builder", 1)
+    try:
+        O1, S1_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt")
+        need1 = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt")
+        with pytest.raises(pf.PfError):
+            pf.pf_set_option("wu_builder", 2)
+    finally:
+        pf.pf_set_option("wu_builder", 0)
+    assert need1 > need0
+    assert util.max_rel(O1.cpu().numpy(), O0.cpu().numpy()) < 2 * util.TOL_F32
+    assert util.max_rel(S1_.cpu().numpy(), S0_.cpu().numpy()) < 2 * util.TOL_F32
