@@ -243,6 +243,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures)")
     ap.add_argument("--heads", type=int, default=0, help="override H of the workload (profiling captures)")
     ap.add_argument("--ring-depth", type=int, default=0, help="pf_set_option('ring_depth', N) before running")
+    ap.add_argument("--segments", type=int, default=0, help="pf_set_option('segments', N) before running")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pf_synth.CONFIGS[args.workload]
@@ -266,6 +267,8 @@ def main():
     import paper_2504_00492_b200 as pf
     if args.ring_depth:
         pf.pf_set_option("ring_depth", args.ring_depth)
+    if args.segments:
+        pf.pf_set_option("segments", args.segments)
     peaks, peak_kind = load_peaks()
 
     host = pf_synth.make_inputs(w, seed=w.seed + 1000 * rank).pin()

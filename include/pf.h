@@ -184,7 +184,17 @@ int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
  *       inverse T' of Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
  *       "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one kernel; it
  *       needs more workspace (pf_workspace_bytes follows the current value).  The tensor-core kernels do not
- *       use it, except PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels. */
+ *       use it, except PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels.
+ *   "segments" (1..64, default 1): with S > 1 every forward call cuts each sequence into S segments of L/S
+ *       tokens and evaluates them side by side (Section 3, "Scan": the flow of an interval is the pair (P, Xi)
+ *       with S_end = S_start P + Xi, Proposition 2.1, and flows of consecutive intervals compose).  Three passes
+ *       over the segments -- from the zero state (gives Xi), from the identity (gives P + Xi), then, after a
+ *       small kernel has composed the S flows of every sequence into the segments' start states, from the true
+ *       start states (gives O) -- so about three times the work, but S times the parallelism: meant for problems
+ *       with far fewer sequences (B*H) than the GPU has SMs.  Needs d_k = d_v and L a multiple of S, otherwise
+ *       the call returns PF_ERR_UNSUPPORTED (and pf_workspace_bytes 0); the workspace grows by four arrays of
+ *       B*H*S*d_k*d_v floats.  A device-side timeout of an earlier pass is overwritten in the status word by
+ *       the next pass on the tensor-core paths. */
 int pf_set_option(const char* name, int value);
 
 /* Number of kernels the last successful call on this host thread enqueued. */

@@ -58,6 +58,7 @@ int check_shape(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
 }
 
 int g_wu_builder = 0;     // option "wu_builder"
+int g_segments = 1;       // option "segments"
 
 Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype) {
     Problem p{};
@@ -117,7 +118,9 @@ bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
     return a0 < b0 + bn && b0 < a0 + an;
 }
 
-int forward(const pf_params* a) {
+// One forward call on the problem as given.  `top`: this is the caller's call itself (it resets and publishes the
+// launch count and the profile list); false for the passes of a segmented call.
+int forward_one(const pf_params* a, bool top) {
     if (!a) return PF_ERR_INVALID;
     int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
     if (st != PF_OK) return st;
@@ -158,8 +161,10 @@ int forward(const pf_params* a) {
         PF_CUDA_TRY(cudaMallocAsync(&ws, need, p.stream));
         own = true;
     }
-    g_launch_accum = 0;
-    g_prof_n = 0;
+    if (top) {
+        g_launch_accum = 0;
+        g_prof_n = 0;
+    }
     const long long rows = (long long)p.B * p.H * p.L * p.r;
     if (a->step == PF_STEP_EXACT && rows > 0) {
         float* b32 = (float*)((uint8_t*)ws + align_up(kernel_workspace_need(p, impl), 256));
@@ -187,8 +192,179 @@ int forward(const pf_params* a) {
         cudaError_t e = cudaFreeAsync(ws, p.stream);
         if (e != cudaSuccess && st == PF_OK) st = record_cuda_error(e, "cudaFreeAsync");
     }
-    if (st == PF_OK) g_launches = g_launch_accum;
+    if (st == PF_OK && top) g_launches = g_launch_accum;
     return st;
+}
+
+// ---- segmented evaluation: the flows of S segments of every sequence in parallel, then their composition --------
+// Section 3, step 3 ("Scan"): the flow of an interval is the pair (P, Xi) with S_end = S_start P + Xi (Proposition 2.1),
+// and flows of consecutive intervals compose.  A sequence of L tokens is cut into S segments of L/S tokens, which the
+// kernels see as S independent sequences (the layout [B,H,L,...] makes that a change of H and L, not a copy):
+//   pass A: every segment from the zero state            -> S_final = Xi_seg
+//   pass B: every segment from the identity (d_v = d_k)  -> S_final = P_seg + Xi_seg   (row j of the state carries e_j P)
+//   compose (one small kernel, serial over the S segments of a sequence, parallel over sequences and rows):
+//           start(0) = S0,  start(s+1) = start(s) P_s + Xi_s;  the last one is S_final
+//   pass C: every segment from its true start state      -> O
+// Three passes instead of one, but each is S times more parallel: worth it when B*H is far below the SM count.
+struct SegArrays {
+    float* xi;      // [B*H*S][d_k][d_v]  pass A's S_final
+    float* pb;      // same, pass B's
+    float* start;   // same, start state of every segment (the S0 of pass C)
+    float* ident;   // same, identity in every slot (the S0 of pass B)
+};
+size_t seg_array_bytes(const pf_params* a, int S) {
+    return align_up((size_t)a->B * a->H * S * a->d_k * a->d_v * sizeof(float), 256);
+}
+
+__global__ void seg_identity_kernel(float* __restrict__ out, long long slots, int d) {
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= slots * d * d) return;
+    const int r = (int)((e / d) % d), c = (int)(e % d);
+    out[e] = r == c ? 1.f : 0.f;
+}
+
+// grid (B*H, d/16), 256 threads; thread (jj, ig): row j = 16*blockIdx.y + jj of the state, columns i = 8*ig .. 8*ig+7.
+// Arrays are in the API layout X[i][j] = S[j][i].
+__global__ void __launch_bounds__(256) seg_compose_kernel(const float* __restrict__ S0, SegArrays arr,
+                                                          float* __restrict__ S_final, int S, int d) {
+    extern __shared__ float sm[];
+    float* Ps = sm;                 // [d][d]   P[i'][i]
+    float* cur = sm + d * d;        // [16][d]  rows of the current state
+    const long long bh = blockIdx.x;
+    const int j0 = blockIdx.y * 16;
+    const int jj = threadIdx.x >> 4, ig = (threadIdx.x & 15) * (d / 16);
+    const int per = d / 16;         // columns per thread: 8 (d = 128) or 4 (d = 64)
+    for (int e = threadIdx.x; e < 16 * d; e += 256) {
+        const int r = e / d, i = e % d;
+        cur[e] = S0 ? S0[(bh * d + i) * d + j0 + r] : 0.f;
+    }
+    __syncthreads();
+    for (int s = 0; s < S; ++s) {
+        const long long slot = bh * S + s;
+        float* st = arr.start + slot * d * d;
+        for (int e = threadIdx.x; e < 16 * d; e += 256) {
+            const int r = e % 16, i = e / 16;
+            st[(long long)i * d + j0 + r] = cur[r * d + i];
+        }
+        const float* xi = arr.xi + slot * d * d;
+        const float* pb = arr.pb + slot * d * d;
+        // P[i'][i] = (P + Xi)[i'][i] - Xi[i'][i], both stored as [i][i']
+        for (int e = threadIdx.x; e < d * d; e += 256) {
+            const int i = e / d, ip = e % d;
+            Ps[ip * d + i] = pb[e] - xi[e];
+        }
+        __syncthreads();
+        float acc[8];
+        for (int c = 0; c < per; ++c) acc[c] = xi[(long long)(ig + c) * d + j0 + jj];
+        for (int ip = 0; ip < d; ++ip) {
+            const float a = cur[jj * d + ip];
+            for (int c = 0; c < per; ++c) acc[c] = fmaf(a, Ps[ip * d + ig + c], acc[c]);
+        }
+        __syncthreads();
+        for (int c = 0; c < per; ++c) cur[jj * d + ig + c] = acc[c];
+        __syncthreads();
+    }
+    if (S_final)
+        for (int e = threadIdx.x; e < 16 * d; e += 256) {
+            const int r = e % 16, i = e / 16;
+            S_final[(bh * d + i) * d + j0 + r] = cur[r * d + i];
+        }
+}
+
+bool seg_applicable(const pf_params* a, int S) {
+    return S > 1 && a->d_k == a->d_v && a->L > 0 && a->L % S == 0;
+}
+pf_params seg_subproblem(const pf_params* a, int S) {
+    pf_params b = *a;
+    b.H = a->H * S;
+    b.L = a->L / S;
+    return b;
+}
+size_t seg_workspace_need(const pf_params* a, int S) {
+    const pf_params b = seg_subproblem(a, S);
+    Problem p = as_problem(b.B, b.H, b.L, b.d_k, b.d_v, b.r, b.chunk, b.in_dtype);
+    p.mode = b.mode;
+    const int impl = select_impl(p, b.impl);
+    if (impl < 0) return 0;
+    return align_up(workspace_need(p, impl), 256) + 4 * seg_array_bytes(a, S);
+}
+
+int forward_segmented(const pf_params* a, int S) {
+    int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
+    if (st != PF_OK) return st;
+    if (!seg_applicable(a, S)) return PF_ERR_UNSUPPORTED;
+    if (!aligned16(a->S0) || !aligned16(a->S_final)) return PF_ERR_ALIGNMENT;
+    pf_params sub = seg_subproblem(a, S);
+    const size_t need = seg_workspace_need(a, S);
+    if (need == 0) return PF_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)a->stream;
+    void* ws = a->workspace;
+    bool own = false;
+    if (ws) {
+        if (a->workspace_bytes < need || ((uintptr_t)ws & 255u)) return PF_ERR_WORKSPACE;
+    } else {
+        PF_CUDA_TRY(cudaMallocAsync(&ws, need, stream));
+        own = true;
+    }
+    const size_t ab = seg_array_bytes(a, S);
+    uint8_t* tail = (uint8_t*)ws + (need - 4 * ab);
+    SegArrays arr{(float*)tail, (float*)(tail + ab), (float*)(tail + 2 * ab), (float*)(tail + 3 * ab)};
+    sub.workspace = ws;
+    sub.workspace_bytes = need - 4 * ab;
+    g_launch_accum = 0;
+    g_prof_n = 0;
+    const int d = a->d_k;
+    const long long slots = (long long)a->B * a->H * S;
+    auto finish = [&](int code) {
+        if (own) cudaFreeAsync(ws, stream);
+        return code;
+    };
+    // pass A: zero start
+    sub.S0 = nullptr;
+    sub.S_final = arr.xi;
+    st = forward_one(&sub, false);
+    if (st != PF_OK) return finish(st);
+    // pass B: identity start
+    {
+        const long long total = slots * d * d;
+        prof_begin("seg_identity", stream);
+        seg_identity_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(arr.ident, slots, d);
+        prof_end(stream);
+        count_launch();
+    }
+    sub.S0 = arr.ident;
+    sub.S_final = arr.pb;
+    st = forward_one(&sub, false);
+    if (st != PF_OK) return finish(st);
+    // composition of the S flows of every sequence
+    {
+        const int smem = (d * d + 16 * d) * (int)sizeof(float);
+        cudaError_t e = cudaFuncSetAttribute(seg_compose_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_compose_kernel attribute"));
+        prof_begin("seg_compose", stream);
+        seg_compose_kernel<<<dim3((unsigned)(a->B * a->H), (unsigned)(d / 16)), 256, smem, stream>>>(a->S0, arr, a->S_final, S, d);
+        prof_end(stream);
+        count_launch();
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_compose_kernel"));
+    }
+    // pass C: true start states
+    sub.S0 = arr.start;
+    sub.S_final = nullptr;
+    st = forward_one(&sub, false);
+    if (st != PF_OK) return finish(st);
+    if (own) {
+        cudaError_t e = cudaFreeAsync(ws, stream);
+        if (e != cudaSuccess) return record_cuda_error(e, "cudaFreeAsync");
+    }
+    g_launches = g_launch_accum;
+    return PF_OK;
+}
+
+int forward(const pf_params* a) {
+    if (!a) return PF_ERR_INVALID;
+    if (g_segments > 1) return forward_segmented(a, g_segments);
+    return forward_one(a, true);
 }
 
 }  // namespace
@@ -229,6 +405,13 @@ size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chun
     pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
     const int sel = pf::select_impl(p, impl);
     if (sel < 0) return 0;
+    if (pf::g_segments > 1) {
+        pf_params a;
+        memset(&a, 0, sizeof(a));
+        a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
+        a.in_dtype = in_dtype; a.impl = impl;
+        return pf::seg_applicable(&a, pf::g_segments) ? pf::seg_workspace_need(&a, pf::g_segments) : 0;
+    }
     return pf::workspace_need(p, sel);
 }
 
@@ -242,6 +425,11 @@ int pf_last_launch_count(void) { return pf::g_launches; }
 
 int pf_set_option(const char* name, int value) {
     if (!name) return PF_ERR_INVALID;
+    if (strcmp(name, "segments") == 0) {
+        if (value < 1 || value > 64) return PF_ERR_INVALID;
+        pf::g_segments = value;
+        return PF_OK;
+    }
     if (strcmp(name, "wu_builder") == 0) {
         if (value != 0 && value != 1) return PF_ERR_INVALID;
         pf::g_wu_builder = value;

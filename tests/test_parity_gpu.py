@@ -424,3 +424,65 @@ def test_the_two_builders_agree_closely_and_the_option_is_checked():
     assert need1 > need0
     assert util.max_rel(O1.cpu().numpy(), O0.cpu().numpy()) < 2 * util.TOL_F32
     assert util.max_rel(S1_.cpu().numpy(), S0_.cpu().numpy()) < 2 * util.TOL_F32
+
+
+# --- segments evaluated side by side, flows composed (option "segments") -----------------------------------------------
+
+SEGMENT_CASES = [
+    (Workload("sg_simt_f32", B=1, H=2, L=256, d_k=64, d_v=64, r=2, chunk=32, s0_std=0.1, seed=61, dtype="f32"), "simt", 4),
+    (Workload("sg_simt_r3", B=2, H=1, L=120, d_k=128, d_v=128, r=3, chunk=16, beta_scale=2.0, seed=62, dtype="f32"), "simt", 3),
+    (Workload("sg_fused", B=1, H=2, L=2048, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=63), "tc", 8),
+    (Workload("sg_fused_ragged", B=1, H=1, L=1000, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=64), "tc", 2),
+    (Workload("sg_split_d64", B=1, H=2, L=512, d_k=64, d_v=64, r=4, chunk=32, beta_scale=2.0, seed=65), "tc_split", 4),
+]
+
+
+@pytest.fixture
+def segments():
+    import paper_2504_00492_b200 as pf
+
+    def set_(n):
+        pf.pf_set_option("segments", n)
+    yield set_
+    pf.pf_set_option("segments", 1)
+
+
+@pytest.mark.parametrize("w,impl,S", SEGMENT_CASES, ids=lambda x: getattr(x, "name", x))
+def test_segmented_evaluation(segments, w, impl, S):
+    segments(S)
+    if impl == "simt":
+        util.check_parity(w, impl=impl)
+    else:
+        eo, es = _run_with_status(w, impl)
+        assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+
+
+def test_segmented_product_form_exact_step_and_plain_entry_point(segments):
+    import paper_2504_00492_b200 as pf
+    segments(4)
+    w = Workload("sg_modes", B=1, H=2, L=512, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=66)
+    eo, es = _run_with_status(w, "tc", mode="product", step="exact")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)      # library-owned workspace
+    O_ref, Sf_ref = util.run_oracle(inp)
+    assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16 and util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
+
+
+def test_segments_that_do_not_fit_are_refused(segments):
+    import paper_2504_00492_b200 as pf
+    segments(4)
+    w = SMALL[0]                                   # d_k != d_v
+    d = pf_synth.make_inputs(w).to("cuda")
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    assert e.value.status == -2
+    w2 = Workload("sg_bad_L", B=1, H=1, L=130, d_k=64, d_v=64, r=1, chunk=32, seed=67)     # 130 % 4 != 0
+    d2 = pf_synth.make_inputs(w2).to("cuda")
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk)
+    assert e.value.status == -2
+    assert pf.pf_workspace_bytes(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, 0, "auto") == 0
+    with pytest.raises(pf.PfError):
+        pf.pf_set_option("segments", 0)
