@@ -180,6 +180,8 @@ int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
  * PF_ERR_UNSUPPORTED for an unknown name, PF_ERR_INVALID for a value out of range.
  *   "ring_depth" (3..64, default 8): slots per sequence of the L2-resident ring through which the
  *       single-launch tensor-core path hands each chunk's flow to the state scan.
+ *   "flow_ctas" (0..1024, default 0 = no limit): upper limit on the CTAs of the single-launch path that build
+ *       flows (the others scan); for measuring how the time scales with them.
  *   "wu_builder" (0 or 1, default 0): how the fp32 SIMT kernels obtain W and Uh of a chunk.  0: the triangular
  *       inverse T' of Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
  *       "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one kernel; it

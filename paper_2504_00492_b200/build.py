@@ -29,19 +29,20 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ and link libpf.so.  Returns the library path."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str = None) -> str:
+    """Compile every .cu under csrc/ and link libpf.so.  Returns the library path.
+    extra_flags / out: a diagnostic build (e.g. ("-DPF_ENDS",)) into another file, objects kept apart."""
+    if out is None and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     objs = []
-    bdir = os.path.join(PKG, "_build")
+    bdir = os.path.join(PKG, "_build" if out is None else "_build_diag")
     os.makedirs(bdir, exist_ok=True)
     procs = []
     for src in sources():
         obj = os.path.join(bdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *extra_flags, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -49,10 +50,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src, pr in procs:
         if pr.wait() != 0:
             raise RuntimeError(f"nvcc failed on {src}")
-    tmp = LIB + ".tmp%d" % os.getpid()
+    target = LIB if out is None else out
+    tmp = target + ".tmp%d" % os.getpid()
     subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp, *objs], check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":

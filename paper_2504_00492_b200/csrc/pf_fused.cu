@@ -1069,6 +1069,9 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base_s;
+#ifdef PF_ENDS   // diagnostic builds: start and end of every CTA (globaltimer), words 0.. and 160.. of the timing block
+    if (tid == 0) ((unsigned long long*)(ws.status + 256))[blockIdx.x] = globaltimer_ns();
+#endif
 
     if (is_scan) scan_role(g, ws, S0, O, S_final, smem, bar, tb, (int)blockIdx.x);
     else flow_role<N>(maps, g, ws, beta, O, smem, bar, tb, (int)blockIdx.x - g.n_scan);
@@ -1076,6 +1079,9 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
 
     tc_fence_before();
     __syncthreads();
+#ifdef PF_ENDS
+    if (tid == 0) ((unsigned long long*)(ws.status + 256))[160 + blockIdx.x] = globaltimer_ns();
+#endif
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
@@ -1119,6 +1125,7 @@ int sm_count() {
 }
 
 int g_ring_depth = 8;     // slots per sequence (option "ring_depth", 3..64)
+int g_flow_ctas = 0;      // upper limit on flow CTAs (option "flow_ctas"; 0 = every SM that is not scanning)
 
 int ring_depth(const Problem& p) {
     const int NC = p.chunks_per_seq();
@@ -1144,6 +1151,11 @@ Carve carve(const Problem& p) {
 }  // namespace
 
 int fused_set_option(const char* name, int value) {
+    if (strcmp(name, "flow_ctas") == 0) {
+        if (value < 0 || value > 1024) return PF_ERR_INVALID;
+        g_flow_ctas = value;
+        return PF_OK;
+    }
     if (strcmp(name, "ring_depth") == 0) {
         if (value < 3 || value > 64) return PF_ERR_INVALID;
         g_ring_depth = value;
@@ -1183,6 +1195,7 @@ int fused_forward(const Problem& p, void* workspace) {
     const int sms = sm_count();
     g.n_scan = nseq;
     g.n_flow = sms - nseq;
+    if (g_flow_ctas > 0 && g_flow_ctas < g.n_flow) g.n_flow = g_flow_ctas;
     if (g.items < g.n_flow) g.n_flow = g.items > 0 ? g.items : 1;
     FusedMaps maps;
     if (NC > 0) {

@@ -268,6 +268,23 @@ def test_set_option_rejects_bad_input():
     with pytest.raises(pf.PfError) as ei:
         pf.pf_set_option("no_such_option", 1)
     assert ei.value.status == -2
+    with pytest.raises(pf.PfError) as ei:
+        pf.pf_set_option("flow_ctas", -1)
+    assert ei.value.status == -1
+
+
+def test_flow_cta_limit_does_not_change_the_result():
+    import paper_2504_00492_b200 as pf
+    w = FUSED_CASES[0]
+    d = pf_synth.make_inputs(w).to("cuda")
+    O0, S0_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
+    try:
+        for n in (1, 7, 40):
+            pf.pf_set_option("flow_ctas", n)
+            O1, S1_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
+            assert torch.equal(O0, O1) and torch.equal(S0_, S1_)
+    finally:
+        pf.pf_set_option("flow_ctas", 0)
 
 
 def test_back_to_back_launches_without_synchronisation():
