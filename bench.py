@@ -165,6 +165,11 @@ class ClockSampler:
         return out
 
 
+def fwd_of(pf, w):
+    """The entry point for the workload's input type (config 0 is fp32, the others bf16)."""
+    return pf.pf_deltanet_fwd_f32 if w.dtype == "f32" else pf.pf_deltanet_fwd
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -220,7 +225,7 @@ def kernel_profile(pf, d, w, steps):
     lib.pf_profile_enable(1)
     acc = {}
     for _ in range(steps):
-        pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+        fwd_of(pf, w)(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
         torch.cuda.synchronize()
         n = lib.pf_profile_count()
         for i in range(n):
@@ -278,7 +283,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk, O=O, S_final=Sf)
+        fwd_of(pf, w)(d.q, d.k, d.v, d.beta, d.S0, w.chunk, O=O, S_final=Sf)
 
     def barrier():
         if use_dist:
@@ -318,7 +323,7 @@ def main():
 
     def e2e_step():
         dd = host.to("cuda", non_blocking=True)
-        o, s = pf.pf_deltanet_fwd(dd.q, dd.k, dd.v, dd.beta, dd.S0, w.chunk, O=O, S_final=Sf)
+        o, s = fwd_of(pf, w)(dd.q, dd.k, dd.v, dd.beta, dd.S0, w.chunk, O=O, S_final=Sf)
         hO.copy_(o, non_blocking=True)
         hS.copy_(s, non_blocking=True)
 

@@ -83,7 +83,11 @@ enum { PF_MODE_SUM = 0, PF_MODE_PRODUCT = 1 };
 enum { PF_STEP_EULER = 0, PF_STEP_EXACT = 1 };
 
 /* Which kernels evaluate the chunk form.
- *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.
+ *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.  The result does
+ *                  not depend on the chunk length beyond rounding, so AUTO may evaluate with another supported
+ *                  chunk length than the one passed when that puts the problem on the tensor-core kernels (64 or
+ *                  128 rows per chunk: e.g. r = 4 with chunk 64 runs as chunk 32).  The explicit choices below
+ *                  use `chunk` as given.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
  *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.  For
  *                  d_k = d_v = 128 with at most (SM count - 8) sequences this is ONE cooperative launch in

@@ -68,8 +68,22 @@ Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
     return p;
 }
 
-int select_impl(const Problem& p, int impl) {
+// Picks the kernels.  The result of the operation does not depend on the chunk length (beyond rounding), so
+// PF_IMPL_AUTO may replace p.chunk by another supported length when that is what puts the problem on the tensor-core
+// kernels (they take 64 or 128 rows per chunk): config 3 with chunk 64 has 256 rows and would otherwise run on the
+// fp32 kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
+int select_impl(Problem& p, int impl) {
     if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
+    if (impl == PF_IMPL_AUTO && !tc_supported(p)) {
+        for (int c : {64, 32, 16}) {
+            Problem t = p;
+            t.chunk = c;
+            if (tc_supported(t)) {
+                p.chunk = c;
+                break;
+            }
+        }
+    }
     switch (impl) {
         case PF_IMPL_SIMT: return PF_IMPL_SIMT;
         case PF_IMPL_TC: return tc_supported(p) ? (int)PF_IMPL_TC : (int)PF_ERR_UNSUPPORTED;
@@ -418,7 +432,8 @@ size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chun
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
     const int st = pf::check_shape(B, H, L, d_k, d_v, r, chunk);
     if (st != PF_OK) return st;
-    return pf::select_impl(pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype), impl);
+    pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
+    return pf::select_impl(p, impl);
 }
 
 int pf_last_launch_count(void) { return pf::g_launches; }

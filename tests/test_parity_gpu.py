@@ -503,3 +503,24 @@ def test_segments_that_do_not_fit_are_refused(segments):
     assert pf.pf_workspace_bytes(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, 0, "auto") == 0
     with pytest.raises(pf.PfError):
         pf.pf_set_option("segments", 0)
+
+
+# --- PF_IMPL_AUTO may evaluate with another chunk length to reach the tensor-core kernels ---------------------------------
+
+def test_auto_rechunks_onto_the_tensor_core_path():
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    # config 3's shape class: r = 4 with chunk 64 is 256 rows per chunk; chunk 32 gives the 128 the kernels take
+    w = Workload("auto_r4_c64", B=2, H=2, L=500, d_k=64, d_v=64, r=4, chunk=64, beta_scale=2.0, s0_std=0.1, seed=71)
+    assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
+    assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "tc") == -2
+    util.check_parity(w, impl="auto")
+    eo, es = _run_with_status(w, "auto")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+    # r = 1 with chunk 32 is 32 rows: chunk 64 gives 64
+    w2 = Workload("auto_r1_c32", B=1, H=2, L=300, d_k=128, d_v=128, r=1, chunk=32, s0_std=0.1, seed=72)
+    assert pf.pf_select_impl(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
+    util.check_parity(w2, impl="auto")
+    # r = 3 never gives 64 or 128 rows: fp32 kernels, at the caller's chunk length
+    w3 = SMALL[2]
+    assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_SIMT
