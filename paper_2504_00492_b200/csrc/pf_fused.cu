@@ -186,6 +186,24 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
+// Diagnostic builds (-DPF_DELAY_SITE=n [-DPF_DELAY_CLK=c]): the threads that pass site n spin for c cycles (2000 by
+// default) every time.  How much of an injected delay shows up in the kernel time says whether the site is on the
+// critical cycle of the pipeline (about 100 %) or has slack (about 0 %).  Compiled out otherwise.
+#ifdef PF_DELAY_SITE
+#ifndef PF_DELAY_CLK
+#define PF_DELAY_CLK 2000
+#endif
+#define PF_DELAY(site)                                                  \
+    do {                                                                \
+        if ((site) == PF_DELAY_SITE) {                                  \
+            const long long t_ = clock64();                             \
+            while (clock64() - t_ < PF_DELAY_CLK) { }                   \
+        }                                                               \
+    } while (0)
+#else
+#define PF_DELAY(site) do { } while (0)
+#endif
+
 #define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code)
 
 // byte offset of the 16-byte chunk `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
@@ -383,6 +401,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 }
             }
             tc_fence_before();
+            PF_DELAY(0);
             mbar_arrive(&bar[B_GFREE]);
             named_bar(1, 128);
             PF_LAP(1);
@@ -427,6 +446,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             merge_level<N, 32>(x_b, sX, warp, lane);
             if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
             fence_async_smem();
+            PF_DELAY(1);
             mbar_arrive(&bar[B_XREADY + b]);
             PF_LAP(3);
         }
@@ -472,10 +492,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
+            PF_DELAY(2);
             mbar_arrive(&bar[B_WUREADY]);
             PF_LAP(1);
             // ---- conversions for chunk k+1
             if (k + 1 < nk) {
+                PF_DELAY(4);
                 if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
                 PF_LAP(2);
                 cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
@@ -490,6 +512,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 PF_LAP(5);
             }
             // ---- RA = [E | Xi^T], second half: row j = m of Xi^T, one 16-byte piece per column group, into the ring
+            PF_DELAY(3);
             if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
             tc_fence_after();
             PF_LAP(6);
@@ -564,6 +587,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
+            PF_DELAY(5);
             mbar_arrive(&bar[B_WUREADY]);
             PF_LAP(1);
             // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
@@ -591,9 +615,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
+            PF_DELAY(6);
             mbar_arrive(&bar[B_PTREADY]);
             PF_LAP(2);
             // ---- RA = [E | Xi^T], first half: row i of E, one 16-byte piece per column group, into the ring
+            PF_DELAY(7);
             if (!PF_WAIT(B_SLOTOK, k & 1, 121) || !PF_WAIT(B_RADONE, k & 1, 123)) return;
             tc_fence_after();
             PF_LAP(3);
@@ -647,10 +673,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 }
             }
             tc_fence_before();
+            PF_DELAY(8);
             mbar_arrive(&bar[B_D4FREE]);
             mbar_arrive(&bar[B_OUTDONE]);
             PF_LAP(6);
             // ---- Q of the next chunk: convert in place, then take this thread's column
+            PF_DELAY(9);
             if (k + 1 < nk && !q_prepare(k + 1)) return;
             PF_LAP(7);
         }
@@ -664,6 +692,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 int seq, c;
                 item(j, seq, c);
                 // K and V: their regions were last read by the MMAs of chunk j-2
+                PF_DELAY(14);
                 if (j >= 2 && !PF_WAIT(B_D4DONE, (j - 2) & 1, 131)) return;
                 mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
                 for (int h = 0; h < 2; ++h)
@@ -699,6 +728,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 if (k >= 1 && !PF_WAIT(B_RAFREE, (k - 1) & 1, 144)) return;
                 tc_fence_after();
                 PF_LAP(0);
+                PF_DELAY(10);
                 gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
                 commit_uni(&bar[B_D2DONE]);
                 PF_LAP(1);
@@ -707,6 +737,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
                     tc_fence_after();
                     const uint32_t k1_b = smem_u32(smem + b1 * F_REGION + K_OFF);
+                    PF_DELAY(13);
                     gemm_uni<false, false, N, DK, N, N, true>(RG, k1_b, k1_b);
                     commit_uni(&bar[B_GDONE]);
                 }
@@ -722,6 +753,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
                 tc_fence_after();
                 PF_LAP(4);
+                PF_DELAY(11);
                 gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
                 gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
                 commit_uni(&bar[B_RADONE]);
@@ -730,6 +762,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
                 tc_fence_after();
                 PF_LAP(6);
+                PF_DELAY(12);
                 gemm_uni<true, true, 64, N, N, N>(RC, x_b, pt_b);
                 gemm_uni<true, true, 64, N, N, N>(RD, v_b, pt_b);
                 commit_uni(&bar[B_D4DONE]);
@@ -752,6 +785,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 if (!PF_WAIT(B_OUTDONE, k & 1, 163)) return;
                 PF_LAP(1);
                 __threadfence();
+                PF_DELAY(15);
                 st_release_gpu(&ws.ready[seq * 64 + slot_i], c + 1);
                 PF_LAP(2);
             }
@@ -805,6 +839,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             PF_STAMP(1 + 10 * w);
             {
                 uint32_t pk[32];
+                PF_DELAY(16);
 #pragma unroll
                 for (int q = 0; q < 32; ++q) pk[q] = pack_h2(S[2 * q], S[2 * q + 1]);
                 tmem_st32(t_a + buf * 64 + 32 * w + lane_base, pk);

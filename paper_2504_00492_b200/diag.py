@@ -3,6 +3,9 @@
     python -m paper_2504_00492_b200.diag build       # once, anywhere nvcc is: libpf_diag.so with -DPF_ENDS
     python -m paper_2504_00492_b200.diag ends         # when each CTA of one launch starts and ends (device clock)
     python -m paper_2504_00492_b200.diag flow-ctas    # time per call against the number of flow-building CTAs
+    python -m paper_2504_00492_b200.diag build-delays # anywhere nvcc is: 17 libraries, each with a 2000-cycle spin at
+                                                      # one hand-off of the pipeline (-DPF_DELAY_SITE=n)
+    python -m paper_2504_00492_b200.diag sensitivity  # time per call of each of them against the ordinary library
 
 `ends` needs the diagnostic library (thread 0 of every CTA stamps the global timer into the status block of the
 workspace); `flow-ctas` runs on the ordinary library through pf_set_option("flow_ctas", n)."""
@@ -77,6 +80,65 @@ def flow_ctas():
         pf.pf_set_option("flow_ctas", 0)
 
 
+DELAY_SITES = {
+    0: "solve warps, after the Gram epilogue", 1: "solve warps, after the inverse (before X is ready)",
+    2: "mid warps, after the Uh epilogue", 3: "mid warps, before the Xi^T drain", 4: "mid warps, before converting V",
+    5: "out warps, after the W epilogue", 6: "out warps, after the P^T epilogue", 7: "out warps, before the E drain",
+    8: "out warps, after the Qt / OI drain", 9: "out warps, before preparing Q", 10: "MMA warp, before [Uh|W] = X [V|K]",
+    11: "MMA warp, before E and Xi^T", 12: "MMA warp, before Qt^T and OI^T", 13: "MMA warp, before the next Gram product",
+    14: "TMA warp, before loading K", 15: "flag warp, before the release of the ready flag",
+    16: "scan CTAs: chain warps, before publishing the state (128 steps per sequence)",
+}
+
+
+def _delay_lib(site: int) -> str:
+    return os.path.join(PKG, "_build_diag", f"libpf_delay{site}.so")
+
+
+def build_delays():
+    """Only pf_fused.cu differs between the variants: its object is rebuilt, the others come from the ordinary build."""
+    import glob
+    import subprocess
+    sys.path.insert(0, os.path.dirname(PKG))
+    from paper_2504_00492_b200 import build as _b
+    _b.build()
+    others = [o for o in glob.glob(os.path.join(PKG, "_build", "*.o")) if os.path.basename(o) != "pf_fused.o"]
+    os.makedirs(os.path.join(PKG, "_build_diag"), exist_ok=True)
+    procs = []
+    for site in DELAY_SITES:
+        obj = os.path.join(PKG, "_build_diag", f"pf_fused_delay{site}.o")
+        cmd = ["nvcc", *_b.NVCC_FLAGS, f"-DPF_DELAY_SITE={site}", "-I", os.path.join(_b.ROOT, "include"), "-I", _b.CSRC,
+               "-c", os.path.join(_b.CSRC, "pf_fused.cu"), "-o", obj]
+        procs.append((site, obj, subprocess.Popen(cmd)))
+        if len(procs) % 6 == 0:
+            for _, _, pr in procs[-6:]:
+                pr.wait()
+    for site, obj, pr in procs:
+        if pr.wait() != 0:
+            raise RuntimeError(f"nvcc failed for site {site}")
+        subprocess.run(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", _delay_lib(site), obj,
+                        *others], check=True)
+    print("built", len(procs), "libraries under", os.path.join(PKG, "_build_diag"))
+
+
+def sensitivity():
+    """Each variant in a process of its own (one library per process)."""
+    import subprocess
+    def run(lib):
+        code = ("import sys; sys.argv=['x']; from paper_2504_00492_b200 import diag; "
+                f"t,pf,w,ws,call = diag._setup({lib!r}); print(diag._time(t, call))")
+        out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, cwd=os.path.dirname(PKG))
+        return float(out.stdout.strip().splitlines()[-1])
+    base = sorted(run(None) for _ in range(3))[1]
+    print(f"ordinary library: {base:.1f} us per call (median of 3)")
+    for site, name in DELAY_SITES.items():
+        us = run(_delay_lib(site))
+        per = 128 if site == 16 else 36       # delays per CTA: chunks per flow CTA / steps per scan CTA at config 2
+        injected = per * 2000 / 1965.0
+        print(f"site {site:2d} {name:62s}: {us:6.1f} us  +{us - base:5.1f} us = {100 * (us - base) / injected:4.0f} % of "
+              f"the {injected:.0f} us injected")
+
+
 if __name__ == "__main__":
     what = sys.argv[1] if len(sys.argv) > 1 else ""
     if what == "build":
@@ -87,5 +149,9 @@ if __name__ == "__main__":
         ends()
     elif what == "flow-ctas":
         flow_ctas()
+    elif what == "build-delays":
+        build_delays()
+    elif what == "sensitivity":
+        sensitivity()
     else:
         raise SystemExit(__doc__)
