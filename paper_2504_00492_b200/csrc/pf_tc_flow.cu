@@ -39,15 +39,22 @@ struct FlowSmem {
     static constexpr int w_bytes = (DK / 64) * N * 128;
     static constexpr int pt_bytes = N * 128;                      // P^T: [n rows m][64 cols t]
     static constexpr int id_bytes = 64 * 128;                     // 64 x 64 identity
+    // Two regions are borrowed instead of owned: the identity lives in the X region, which is dead once the W / Uh
+    // product has read X (it is rewritten there for every chunk), and the fp32 diagonal blocks of the inverse live
+    // in the W region, which is written only after the inverse is complete.  With d_k = d_v = 64 that brings a CTA
+    // under half an SM's shared memory, and with the 256 tensor-memory columns those shapes need, two CTAs share an SM.
+    static constexpr bool two_per_sm = (DK + DV <= 128) && (N + 64 <= 256);
+    static constexpr int tmem_cols = two_per_sm ? 256 : 512;
     static constexpr int kq_off = 0;
     static constexpr int v_off = kq_off + kq_bytes;
     static constexpr int x_off = v_off + v_bytes;
     static constexpr int w_off = x_off + x_bytes;
     static constexpr int pt_off = w_off + w_bytes;
-    static constexpr int id_off = pt_off + pt_bytes;
-    static constexpr int diag_off = id_off + id_bytes;            // fp32 [N/16][16][16]
+    static constexpr int id_off = x_off;                          // (borrowed, see above)
+    static constexpr int diag_off = w_off;                        // fp32 [N/16][16][16] (borrowed)
     static constexpr int diag_bytes = (N / 16) * 256 * 4;
-    static constexpr int beta_off = diag_off + diag_bytes;        // fp16 beta[N] (column scaling)
+    static_assert(id_bytes <= x_bytes && diag_bytes <= w_bytes, "borrowed regions fit");
+    static constexpr int beta_off = pt_off + pt_bytes;            // fp16 beta[N] (column scaling)
     static constexpr int total = beta_off + 1024;
 };
 
@@ -126,7 +133,7 @@ __device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, 
 }
 
 template <int N, int DK, int DV>
-__global__ void __launch_bounds__(FLOW_THREADS, 1)
+__global__ void __launch_bounds__(FLOW_THREADS, (FlowSmem<N, DK, DV>::two_per_sm ? 2 : 1))
 tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bfloat16* __restrict__ beta,
         float* __restrict__ O, long long G, int dvs) {
     using SM = FlowSmem<N, DK, DV>;
@@ -159,21 +166,18 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         prefetch_tmap(&maps.v);
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(&tmem_base_s, 512);
-    // 64 x 64 identity, fp16, slab layout; the Q rows of the KQ slabs start defined (stale rows are read)
-    for (int e = tid; e < 64 * 8; e += FLOW_THREADS) {
-        const int row = e >> 3, ch = e & 7;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if ((row >> 3) == ch) ((uint16_t*)&val)[row & 7] = 0x3C00;   // 1.0 in fp16
-        *(uint4*)(sI + row * 128 + ((ch ^ (row & 7)) << 4)) = val;
-    }
+    if (warp == 0) tmem_alloc(&tmem_base_s, SM::tmem_cols);
+    // (the Q rows of the KQ slabs start defined: stale rows are read)
     for (int e = tid; e < SM::kq_bytes / 16; e += FLOW_THREADS) ((uint4*)sKQ)[e] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base_s;
-    const uint32_t t_d1 = tb, t_d2 = tb + 256, t_d3 = tb, t_d4 = tb + 256;
+    // [G | P0^T] (N + 64 columns), then [W | Uh], then [E | Xi] next to [Qt^T | O_intra^T]; each is drained before the
+    // next product that reuses its columns is issued
+    const uint32_t t_d1 = tb, t_d2 = SM::two_per_sm ? tb : tb + 256, t_d3 = SM::two_per_sm ? tb + 128 : tb,
+                   t_d4 = SM::two_per_sm ? tb : tb + 256;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     uint32_t tma_phase = 0, mma_phase = 0;
     bool ok = true;
@@ -357,6 +361,13 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         tc_fence_after();
 
         lap(7);
+        // 64 x 64 identity, fp16, slab layout, into the (now dead) X region: B operand of the "+ Q^T" product below
+        for (int e = tid; e < 64 * 8; e += FLOW_THREADS) {
+            const int row = e >> 3, ch = e & 7;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if ((row >> 3) == ch) ((uint16_t*)&val)[row & 7] = 0x3C00;   // 1.0 in fp16
+            *(uint4*)(sI + row * 128 + ((ch ^ (row & 7)) << 4)) = val;
+        }
         // ---- epilogue 2: W and Uh as fp16 operands (Uh overwrites V) ----------------------------------
 #pragma unroll 1
         for (int c0 = 0; c0 < DK + DV; c0 += 32) {
@@ -460,7 +471,7 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 512);
+    if (warp == 0) tmem_dealloc(tb, SM::tmem_cols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -502,7 +513,8 @@ int launch(const Problem& p, const TcWs& ws, int dvs, const FlowMaps& maps) {
     PF_CUDA_TRY(cudaGetDevice(&dev));
     PF_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const long long G = p.total_chunks();
-    const unsigned grid = (unsigned)(G < sms ? G : sms);
+    const long long slots = (long long)sms * (SM::two_per_sm ? 2 : 1);
+    const unsigned grid = (unsigned)(G < slots ? G : slots);
     prof_begin("tc_flow", p.stream);
     tc_flow<N, DK, DV><<<grid, FLOW_THREADS, smem, p.stream>>>(maps, tc_geo(p), ws, (const __nv_bfloat16*)p.beta, p.O, G, dvs);
     prof_end(p.stream);
