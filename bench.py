@@ -65,7 +65,7 @@ def flops_per_chunk(w, tri: bool) -> dict:
 
 # DRAM bytes (read + write) of one launch of the single-launch kernel from an ncu capture, valid only for the
 # kernel sources it was taken on (their hash is stored with it): {workload: (sha256 of the sources, bytes)}.
-NCU_TRAFFIC = {"c2": ("7231a5c815cd7dd3", 338708224 + 126748672)}
+NCU_TRAFFIC = {"c2": ("63b2cbe9ed107556", 337494016 + 125681408)}
 
 
 def kernel_source_hash() -> str:

@@ -92,7 +92,8 @@ enum { PF_STEP_EULER = 0, PF_STEP_EXACT = 1 };
  *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.  For
  *                  d_k = d_v = 128 with at most (SM count - 8) sequences this is ONE cooperative launch in
  *                  which flow-building CTAs and state-scanning CTAs run side by side; other shapes take
- *                  the two-launch form below.   */
+ *                  the two-launch form below.  (PF_IMPL_AUTO takes the single launch only up to 0.7 x SM count
+ *                  sequences: beyond that too few SMs are left for building flows and two launches are faster.)   */
 enum { PF_IMPL_AUTO = 0, PF_IMPL_SIMT = 1, PF_IMPL_TC = 2,
        /* diagnostic: per-chunk flows built by the fp32 SIMT kernels, state scan on tensor cores */
        PF_IMPL_TC_REFFLOW = 3,

@@ -74,6 +74,7 @@ Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
 // fp32 kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
 int select_impl(Problem& p, int impl) {
     if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
+    p.auto_impl = impl == PF_IMPL_AUTO;
     if (impl == PF_IMPL_AUTO && !tc_supported(p)) {
         for (int c : {64, 32, 16}) {
             Problem t = p;
@@ -94,9 +95,13 @@ int select_impl(Problem& p, int impl) {
     }
 }
 
+// PF_IMPL_TC: the single launch where it supports the shape; under PF_IMPL_AUTO only where it is also the faster of
+// the two tensor-core forms (an explicit PF_IMPL_TC takes it whenever it can run).
+bool use_fused(const Problem& p) { return fused_supported(p) && (!p.auto_impl || fused_preferred(p)); }
+
 // what the kernels of `impl` carve up (the fp32 step sizes of PF_STEP_EXACT follow it)
 size_t kernel_workspace_need(const Problem& p, int impl) {
-    if (impl == PF_IMPL_TC) return fused_supported(p) ? fused_workspace_bytes(p) : tc_workspace_bytes(p);
+    if (impl == PF_IMPL_TC) return use_fused(p) ? fused_workspace_bytes(p) : tc_workspace_bytes(p);
     if (impl == PF_IMPL_TC_SPLIT) return tc_workspace_bytes(p);
     if (impl == PF_IMPL_TC_REFFLOW) return tc_refflow_workspace_bytes(p);
     return simt_workspace_bytes(p);
@@ -198,7 +203,7 @@ int forward_one(const pf_params* a, bool top) {
         }
         p.beta32 = b32;
     }
-    if (impl == PF_IMPL_TC) st = fused_supported(p) ? fused_forward(p, ws) : tc_forward(p, ws);
+    if (impl == PF_IMPL_TC) st = use_fused(p) ? fused_forward(p, ws) : tc_forward(p, ws);
     else if (impl == PF_IMPL_TC_SPLIT) st = tc_forward(p, ws);
     else if (impl == PF_IMPL_TC_REFFLOW) st = tc_forward_refflow(p, ws);
     else st = simt_forward(p, ws);

@@ -24,6 +24,7 @@ struct Problem {
     int in_dtype;
     int mode;           // PF_MODE_SUM (0) or PF_MODE_PRODUCT
     const float* beta32;    // null, or fp32 step sizes [B,H,L,r] (device) that the kernels use in place of beta
+    bool auto_impl;         // the caller left the choice of kernels to the library (PF_IMPL_AUTO)
     int wu_builder;         // fp32 SIMT path: 0 = triangular inverse then W = T'K, Uh = T'V; 1 = the wavefront system of
                             // Theorem 3.3 (option "wu_builder")
     cudaStream_t stream;

@@ -1199,6 +1199,13 @@ int fused_set_option(const char* name, int value) {
     return PF_ERR_UNSUPPORTED;
 }
 
+// One CTA per sequence scans, the rest build flows.  Measured at d = 128, r = 2: up to about 100 sequences the single
+// launch beats the two-launch form (96: 400 against 477 us at L = 2048), beyond that too few SMs are left for the
+// flows (120: 865 against 600 us; 136: 2194 against 669 us).
+bool fused_preferred(const Problem& p) {
+    return (long long)p.B * p.H * 10 <= (long long)sm_count() * 7;
+}
+
 bool fused_supported(const Problem& p) {
     if (p.in_dtype != PF_DTYPE_BF16 || p.d_k != DK || p.d_v != DV) return false;
     const int n = p.n();

@@ -33,6 +33,7 @@ size_t tc_refflow_workspace_bytes(const Problem& p);
 
 // pf_fused.cu: flow builders and state scan in one cooperative launch
 bool fused_supported(const Problem& p);
+bool fused_preferred(const Problem& p);     // enough SMs are left for building flows that the single launch wins
 size_t fused_workspace_bytes(const Problem& p);
 int fused_forward(const Problem& p, void* workspace);
 int fused_set_option(const char* name, int value);

@@ -524,3 +524,21 @@ def test_auto_rechunks_onto_the_tensor_core_path():
     # r = 3 never gives 64 or 128 rows: fp32 kernels, at the caller's chunk length
     w3 = SMALL[2]
     assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_SIMT
+
+
+def test_auto_leaves_the_single_launch_when_few_sms_remain_for_flows():
+    """Up to 0.7 x SM count sequences PF_IMPL_AUTO takes the single launch, beyond that the two-launch form; an
+    explicit PF_IMPL_TC takes the single launch whenever it can run.  Told apart by the number of kernels launched."""
+    import paper_2504_00492_b200 as pf
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    many = Workload("auto_many_seq", B=4, H=(sms * 8 // 10 + 3) // 4, L=192, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=73)
+    few = many.with_(B=1, H=8)
+    assert many.B * many.H * 10 > sms * 7 and many.B * many.H <= sms - 8
+    for w, impl, launches in ((many, "auto", 2), (many, "tc", 1), (few, "auto", 1)):
+        inp = pf_synth.make_inputs(w)
+        d = inp.to("cuda")
+        O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl)
+        torch.cuda.synchronize()
+        assert pf.pf_last_launch_count() == launches, (w.name, impl, pf.pf_last_launch_count())
+        O_ref, Sf_ref = util.run_oracle(inp)
+        assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16 and util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
