@@ -96,7 +96,7 @@ class ClockSampler:
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int, period_ms: int = 20):
+    def __init__(self, gpu_index: int, period_ms: int = 50):
         self.gpu = gpu_index
         self.period_ms = period_ms
         self.proc = None
@@ -163,6 +163,46 @@ class ClockSampler:
             out.update(sm_mhz=statistics.median(x[1] for x in use), sm_max_mhz=max(x[2] for x in use),
                        reasons=sorted({nm for x in use for nm in x[3]}), samples=len(use), window=window)
         return out
+
+
+class Ranks:
+    """The multi-process plumbing of a replicated run: one process per GPU, no data-path collective (sequences are
+    independent, every rank runs its own replica of the workload on inputs of its own seed).  The only exchanges are
+    the barriers around the timed region and the max over ranks of the measured time."""
+
+    def __init__(self, backend: str = "nccl", device: str = "cuda"):
+        self.rank, self.world, self.local = dist_env()
+        self.device = device
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            kw = {"device_id": torch.device("cuda", self.local)} if backend == "nccl" else {}
+            dist.init_process_group(backend, **kw)
+            self.dist = dist
+
+    def seed(self, base: int) -> int:
+        return base + 1000 * self.rank
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        if self.device == "cuda":
+            torch.cuda.synchronize()
+
+    def max_over_ranks(self, ms: float) -> float:
+        if self.dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=self.device)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def job_value(self, units_per_rank_step: float, steps: int, ms: float) -> float:
+        """Whole-job throughput: what all ranks processed, over the slowest rank's time."""
+        return units_per_rank_step * self.world * steps / (self.max_over_ranks(ms) * 1e-3)
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
 
 
 def fwd_of(pf, w):
@@ -260,14 +300,11 @@ def main():
         run_reference(args, w)
         return
 
-    rank, world, local = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local)
-    use_dist = world > 1
-    if use_dist:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(dist_env()[2])
+    ranks = Ranks("nccl", "cuda")
+    rank, world, local = ranks.rank, ranks.world, ranks.local
 
     import paper_2504_00492_b200 as pf
     if args.ring_depth:
@@ -276,7 +313,7 @@ def main():
         pf.pf_set_option("segments", args.segments)
     peaks, peak_kind = load_peaks()
 
-    host = pf_synth.make_inputs(w, seed=w.seed + 1000 * rank).pin()
+    host = pf_synth.make_inputs(w, seed=ranks.seed(w.seed)).pin()
     d = host.to("cuda")
     O = torch.empty(w.B, w.H, w.L, w.d_v, dtype=torch.float32, device="cuda")
     Sf = torch.empty(w.B, w.H, w.d_k, w.d_v, dtype=torch.float32, device="cuda")
@@ -285,10 +322,7 @@ def main():
     def step():
         fwd_of(pf, w)(d.q, d.k, d.v, d.beta, d.S0, w.chunk, O=O, S_final=Sf)
 
-    def barrier():
-        if use_dist:
-            dist.barrier()
-        torch.cuda.synchronize()
+    barrier = ranks.barrier
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -309,10 +343,7 @@ def main():
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else {}
     total_ms = ev[0].elapsed_time(ev[-1])
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    if use_dist:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = ranks.max_over_ranks(total_ms)
     tokens_per_step = w.tokens * world
     value = tokens_per_step * args.steps / (total_ms * 1e-3)
 
@@ -336,10 +367,7 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if use_dist:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = ranks.max_over_ranks(e2e_ms)
     e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3)
     h2d = host.nbytes()
     d2h = hO.numel() * 4 + hS.numel() * 4
@@ -413,8 +441,7 @@ def main():
             "path_roofline": path, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
-    if use_dist:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 if __name__ == "__main__":
