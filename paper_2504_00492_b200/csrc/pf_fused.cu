@@ -137,73 +137,6 @@ enum {
     B_COUNT = 54
 };
 
-// Diagnostic builds (-DPF_TIMING): chosen threads of flow CTA 0 and of scan CTA 0 accumulate the cycles they
-// spend in each wait (indexed by the wait's code) and in each lap, in the 64-bit words that follow the first
-// 1 KB of the status block.  Otherwise null, and the accounting compiles away.
-__device__ __forceinline__ unsigned long long* timing_slot(const FusedWs& ws, bool chosen) {
-#ifdef PF_TIMING
-    return chosen ? (unsigned long long*)(ws.status + 256) : nullptr;
-#else
-    (void)ws; (void)chosen;
-    return nullptr;
-#endif
-}
-#ifdef PF_TIMING
-#define PF_LAP(id)                                          \
-    do {                                                    \
-        if (tim) {                                          \
-            const long long n_ = clock64();                 \
-            lapacc[(id)] += n_ - t_lap;                     \
-            t_lap = n_;                                     \
-        }                                                   \
-    } while (0)
-#define PF_LAP_FLUSH(role)                                                                              \
-    do {                                                                                                \
-        if (tim)                                                                                        \
-            for (int l_ = 0; l_ < 8; ++l_) atomicAdd(tim + 8 * (role) + l_, (unsigned long long)lapacc[l_]); \
-    } while (0)
-#else
-#define PF_LAP(id) do { } while (0)
-#define PF_LAP_FLUSH(role) do { } while (0)
-#endif
-// Diagnostic builds (-DPF_STAMPS): the clock at each event of scan step PF_STAMP_STEP of sequence 0, written by
-// whole warps (no divergence) into unused shared memory of the scan role and copied to words 320.. of the
-// timing block when the chain ends: the timeline of one step.
-#ifdef PF_STAMPS
-#define PF_STAMP_STEP 64
-#define PF_STAMP_OFF (S_OUT + 2 * 32768)
-#define PF_STAMP(id)                                                                                       \
-    do {                                                                                                   \
-        if (seq == 0 && c == PF_STAMP_STEP) ((volatile uint32_t*)(smem + PF_STAMP_OFF))[(id)] = (uint32_t)clock64(); \
-    } while (0)
-#else
-#define PF_STAMP(id) do { } while (0)
-#endif
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Diagnostic builds (-DPF_DELAY_SITE=n [-DPF_DELAY_CLK=c]): the threads that pass site n spin for c cycles (2000 by
-// default) every time.  How much of an injected delay shows up in the kernel time says whether the site is on the
-// critical cycle of the pipeline (about 100 %) or has slack (about 0 %).  Compiled out otherwise.
-#ifdef PF_DELAY_SITE
-#ifndef PF_DELAY_CLK
-#define PF_DELAY_CLK 2000
-#endif
-#define PF_DELAY(site)                                                  \
-    do {                                                                \
-        if ((site) == PF_DELAY_SITE) {                                  \
-            const long long t_ = clock64();                             \
-            while (clock64() - t_ < PF_DELAY_CLK) { }                   \
-        }                                                               \
-    } while (0)
-#else
-#define PF_DELAY(site) do { } while (0)
-#endif
-
 #define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code)
 
 // byte offset of the 16-byte chunk `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
@@ -314,13 +247,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = g.r, C = g.C, nseq = g.nseq;
     int* err = ws.status;
-    unsigned long long* const tim =
-        timing_slot(ws, fid == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416 || tid == 448));
-    const long long t_role = clock64();
-    const unsigned long long t_ns = tim ? globaltimer_ns() : 0ull;
-    long long t_lap = t_role;
-    long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    (void)t_lap; (void)lapacc;
     const int nk = fid < g.items ? (g.items - fid + g.n_flow - 1) / g.n_flow : 0;
     const uint32_t RA = tb, RG = tb + 256, RC = tb + 384, RD = tb + 448;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -374,7 +300,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             ok = ok && PF_WAIT(B_GDONE, k & 1, 102);
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
-            PF_LAP(0);
             // A = Mstrict (.) (G diag(beta)) as fp16 into X; column groups right of the warp's rows are zero
 #pragma unroll 1
             for (int c0 = 0; c0 < N; c0 += 32) {
@@ -401,10 +326,8 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 }
             }
             tc_fence_before();
-            PF_DELAY(0);
             mbar_arrive(&bar[B_GFREE]);
             named_bar(1, 128);
-            PF_LAP(1);
             // 16x16 diagonal blocks: forward substitution, one thread per column of one block (fp32)
             float x[16];
             const int bk = tid >> 4, cc = tid & 15;
@@ -441,16 +364,12 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     *(__half*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4) + (cc & 7) * 2) = __float2half_rn(x[mm]);
             }
             named_bar(1, 128);
-            PF_LAP(2);
             merge_level<N, 16>(x_b, sX, warp, lane);
             merge_level<N, 32>(x_b, sX, warp, lane);
             if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
             fence_async_smem();
-            PF_DELAY(1);
             mbar_arrive(&bar[B_XREADY + b]);
-            PF_LAP(3);
         }
-        PF_LAP_FLUSH(0);
     } else if (warp < 8) {
         // ------------------------------------------------ mid: Uh and Xi^T halves, conversions of V and K -----
         const int m = tid - 128;
@@ -475,7 +394,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // ---- RA = X [V | K], first half:  Uh = diag(beta) (X V), fp16, over V
             if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
             tc_fence_after();
-            PF_LAP(0);
             {
                 const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
                 uint8_t* sU = smem + b * F_REGION + V_OFF;
@@ -492,30 +410,21 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
-            PF_DELAY(2);
             mbar_arrive(&bar[B_WUREADY]);
-            PF_LAP(1);
             // ---- conversions for chunk k+1
             if (k + 1 < nk) {
-                PF_DELAY(4);
                 if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
-                PF_LAP(2);
                 cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
                 fence_async_smem();
                 mbar_arrive(&bar[B_V16 + b1]);
-                PF_LAP(3);
                 if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
-                PF_LAP(4);
                 cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
                 fence_async_smem();
                 mbar_arrive(&bar[B_K16 + b1]);
-                PF_LAP(5);
             }
             // ---- RA = [E | Xi^T], second half: row j = m of Xi^T, one 16-byte piece per column group, into the ring
-            PF_DELAY(3);
             if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
             tc_fence_after();
-            PF_LAP(6);
             {
                 uint8_t* xrow = slot + SLOT_XI + m * 16;
 #pragma unroll 1
@@ -530,9 +439,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
             mbar_arrive(&bar[B_OUTDONE]);
-            PF_LAP(7);
         }
-        PF_LAP_FLUSH(1);
     } else if (warp < 12) {
         // ------------------------------------------------ out: W half, P^T, E / Qt / OI into the ring, Q ---------
         const int i = tid - 256;
@@ -570,7 +477,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // ---- RA = X [V | K], second half:  -W = -diag(beta) (X K), fp16, over X
             if (!PF_WAIT(B_D2DONE, k & 1, 125)) return;
             tc_fence_after();
-            PF_LAP(0);
             {
                 const float bm = (i < N) ? -sBeta[b * 128 + i] : 0.f;
                 uint8_t* sW = smem + b * F_REGION + X_OFF;
@@ -587,9 +493,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
-            PF_DELAY(5);
             mbar_arrive(&bar[B_WUREADY]);
-            PF_LAP(1);
             // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
             if (k >= 1 && !PF_WAIT(B_D4DONE, (k - 1) & 1, 116)) return;
             if (!PF_WAIT(B_P0DONE, k & 1, 117)) return;
@@ -615,14 +519,10 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             fence_async_smem();
             tc_fence_before();
-            PF_DELAY(6);
             mbar_arrive(&bar[B_PTREADY]);
-            PF_LAP(2);
             // ---- RA = [E | Xi^T], first half: row i of E, one 16-byte piece per column group, into the ring
-            PF_DELAY(7);
             if (!PF_WAIT(B_SLOTOK, k & 1, 121) || !PF_WAIT(B_RADONE, k & 1, 123)) return;
             tc_fence_after();
-            PF_LAP(3);
             {
                 uint8_t* erow = slot + SLOT_E + i * 16;
 #pragma unroll 1
@@ -636,11 +536,9 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
-            PF_LAP(4);
             // ---- RC: Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t] (row i of the Qt image);  RD: OI^T[j][t] -> OI[t][j] (fp32)
             if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
             tc_fence_after();
-            PF_LAP(5);
             {
                 uint8_t* qrow = slot + SLOT_QT + i * 16;
 #pragma unroll
@@ -673,16 +571,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 }
             }
             tc_fence_before();
-            PF_DELAY(8);
             mbar_arrive(&bar[B_D4FREE]);
             mbar_arrive(&bar[B_OUTDONE]);
-            PF_LAP(6);
             // ---- Q of the next chunk: convert in place, then take this thread's column
-            PF_DELAY(9);
             if (k + 1 < nk && !q_prepare(k + 1)) return;
-            PF_LAP(7);
         }
-        PF_LAP_FLUSH(2);
     } else if (warp == 12) {
         // ------------------------------------------------ TMA loads -------------------------------------------
         if (lane == 0) {
@@ -692,7 +585,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 int seq, c;
                 item(j, seq, c);
                 // K and V: their regions were last read by the MMAs of chunk j-2
-                PF_DELAY(14);
                 if (j >= 2 && !PF_WAIT(B_D4DONE, (j - 2) & 1, 131)) return;
                 mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
                 for (int h = 0; h < 2; ++h)
@@ -727,48 +619,35 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     return;
                 if (k >= 1 && !PF_WAIT(B_RAFREE, (k - 1) & 1, 144)) return;
                 tc_fence_after();
-                PF_LAP(0);
-                PF_DELAY(10);
                 gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
                 commit_uni(&bar[B_D2DONE]);
-                PF_LAP(1);
                 // G of the next chunk, from its bf16 tile (RG: the solve warps have drained G of this chunk)
                 if (k + 1 < nk) {
                     if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
                     tc_fence_after();
                     const uint32_t k1_b = smem_u32(smem + b1 * F_REGION + K_OFF);
-                    PF_DELAY(13);
                     gemm_uni<false, false, N, DK, N, N, true>(RG, k1_b, k1_b);
                     commit_uni(&bar[B_GDONE]);
                 }
-                PF_LAP(2);
                 // P0^T = K Q^T   (RC and RD: Qt^T and OI^T of chunk k-1 have been drained)
                 if (!PF_WAIT(B_Q16, k & 1, 148)) return;
                 if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
                 tc_fence_after();
                 gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
                 commit_uni(&bar[B_P0DONE]);
-                PF_LAP(3);
                 // E = K^T (-W)  (lanes i, columns i'),   Xi^T = Uh^T K  (lanes j, columns i)
                 if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
                 tc_fence_after();
-                PF_LAP(4);
-                PF_DELAY(11);
                 gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
                 gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
                 commit_uni(&bar[B_RADONE]);
                 // Qt^T - Q^T = (-W)^T P^T over P0^T (which the out warps have turned into P^T),  OI^T = Uh^T P^T
-                PF_LAP(5);
                 if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
                 tc_fence_after();
-                PF_LAP(6);
-                PF_DELAY(12);
                 gemm_uni<true, true, 64, N, N, N>(RC, x_b, pt_b);
                 gemm_uni<true, true, 64, N, N, N>(RD, v_b, pt_b);
                 commit_uni(&bar[B_D4DONE]);
-                PF_LAP(7);
             }
-            PF_LAP_FLUSH(4);
         }
     } else {
         // ------------------------------------------------ flag warp: ring back-pressure, ready flags ---------
@@ -781,20 +660,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 // the scan must be done with the chunk that used this slot before
                 if (c >= g.R && !flag_wait_ge(&ws.consumed[seq * 32], c - g.R + 1, err, 161)) return;
                 mbar_arrive(&bar[B_SLOTOK]);
-                PF_LAP(0);
                 if (!PF_WAIT(B_OUTDONE, k & 1, 163)) return;
-                PF_LAP(1);
                 __threadfence();
-                PF_DELAY(15);
                 st_release_gpu(&ws.ready[seq * 64 + slot_i], c + 1);
-                PF_LAP(2);
             }
-            PF_LAP_FLUSH(5);
         }
-    }
-    if (tim) {      // whole role, per warp: cycles and nanoseconds
-        atomicAdd(tim + 240 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));
-        atomicAdd(tim + 280 + (threadIdx.x >> 5), (unsigned long long)(globaltimer_ns() - t_ns));
     }
 }
 
@@ -806,12 +676,6 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = g.NC;
     int* err = ws.status;
-    unsigned long long* const tim = timing_slot(ws, seq == 0 && (((tid & 127) == 0 && tid < 384) || tid == 384 || tid == 416));
-    const long long t_role = clock64();
-    const unsigned long long t_ns = tim ? globaltimer_ns() : 0ull;
-    long long t_lap = t_role;
-    long long lapacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    (void)t_lap; (void)lapacc;
     const uint32_t t_delta = tb, t_o = tb + 128, t_a = tb + 256;     // Delta | 2 x O^T | 2 x fp16 state
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
@@ -832,44 +696,30 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             const int buf = c & 1;
             // fp16 copy of the state into tensor memory (A operand of Delta and of O^T): 32 packed columns per thread
             bool ok = true;
-            PF_STAMP(0 + 10 * w);
             if (c >= 2) ok = PF_WAIT(B_S16FREE + buf, ((c >> 1) - 1) & 1, 201);
             tc_fence_after();
-            PF_LAP(0);
-            PF_STAMP(1 + 10 * w);
             {
                 uint32_t pk[32];
-                PF_DELAY(16);
 #pragma unroll
                 for (int q = 0; q < 32; ++q) pk[q] = pack_h2(S[2 * q], S[2 * q + 1]);
                 tmem_st32(t_a + buf * 64 + 32 * w + lane_base, pk);
                 tmem_st_wait();
             }
-            PF_LAP(1);
             tc_fence_before();
             if (!named_bar_and(1, 256, ok)) return;
-            PF_LAP(2);
-            PF_STAMP(2 + 10 * w);
             // warp 0 issues Delta[j][i] = sum_i' S[j][i'] E[i][i']; its completion also releases warp 13, which
             // issues the O^T product of the same copy (so that O^T never sits in front of Delta in the tensor pipe)
             if (warp == 0) {
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                PF_STAMP(3);
                 gemm_ta<L_NSK, DK, DK, 128>(t_delta, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
                 commit_uni(&bar[B_APUB + buf]);
             }
-            PF_LAP(3);
-            PF_STAMP(4 + 10 * w);
             if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
-            PF_LAP(4);
-            PF_STAMP(5 + 10 * w);
             if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
-            PF_LAP(5);
-            PF_STAMP(6 + 10 * w);
             // S += Delta + Xi^T   (row j, columns 64w..64w+63; Xi^T from its column-group image)
             const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + j * 16;
 #pragma unroll
@@ -891,15 +741,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
-            PF_LAP(6);
-            PF_STAMP(7 + 10 * w);
         }
-        PF_LAP_FLUSH(8 + w);
-#ifdef PF_STAMPS
-        if (seq == 0 && tid == 0)
-            for (int i_ = 0; i_ < 48; ++i_)
-                ((unsigned long long*)(ws.status + 256))[320 + i_] = ((volatile uint32_t*)(smem + PF_STAMP_OFF))[i_];
-#endif
         if (S_final)
 #pragma unroll
             for (int ii = 0; ii < 64; ++ii) S_final[sbase + (long long)ii * DV] = S[ii];
@@ -915,7 +757,6 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             const int ob = c & 1;
             const int Cv = min(g.C, g.L - c * g.C);
             float* img = (float*)(smem + S_OUT + ob * 32768);
-            PF_STAMP(20);
             bool ok = PF_WAIT(B_ODONE + ob, (c >> 1) & 1, 212);
             tc_fence_after();
             // the reduction of chunk c-2 has read this image (its issuing thread waits, the rest learn of it here)
@@ -924,8 +765,6 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 ok = ok && smem_wait_ge(vis, c + 1, err, 211);     // (long since true: Qt was loaded after it)
             }
             if (!named_bar_and(2, 128, ok)) break;      // (every thread of the four warps leaves together)
-            PF_LAP(0);
-            PF_STAMP(21);
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
@@ -944,11 +783,8 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 bulk_commit();
                 atomicAdd((int*)odone, 4);       // (a counter, not a barrier: the reporter may lag by any amount)
             }
-            PF_LAP(1);
-            PF_STAMP(22);
         }
         if (tid == 256) bulk_wait_all();
-        PF_LAP_FLUSH(10);
     } else if (warp == 12) {
         // ------------------------------------------------ producer: ring -> shared memory ----------------------
         if (lane == 0) {
@@ -967,41 +803,28 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                 // (the flag of chunk c was acquired by load_e(c))
                 const uint8_t* slot = ring + (size_t)(c % g.R) * SLOT_BYTES;
                 const int b = c & 1;
-                PF_STAMP(30);
                 if (c >= 2 && !PF_WAIT(B_XIEMPTY + b, ((c >> 1) - 1) & 1, 224)) return;
-                PF_STAMP(31);
                 mbar_expect_tx(&bar[B_XIFULL + b], DK * DV * 2);
                 bulk_load(smem + S_XI + b * 32768, slot + SLOT_XI, DK * DV * 2, &bar[B_XIFULL + b]);
-                PF_LAP(0);
                 if (c >= 2 && !PF_WAIT(B_QTEMPTY + b, ((c >> 1) - 1) & 1, 223)) return;
-                PF_STAMP(32);
                 mbar_expect_tx(&bar[B_QTFULL + b], DK * 128);
                 bulk_load(smem + S_QT + b * 16384, slot + SLOT_QT, DK * 128, &bar[B_QTFULL + b]);
-                PF_LAP(1);
                 if (c + 1 < NC && !load_e(c + 1)) return;
-                PF_LAP(2);
-                PF_STAMP(33);
             }
-            PF_LAP_FLUSH(11);
         }
     } else if (warp == 13) {
         // ------------------------------------------------ O^T[j][t] = sum_i S[j][i] Qt^T[i][t] (whole warp) -----
 #pragma unroll 1
         for (int c = 0; c < NC; ++c) {
             const int buf = c & 1;
-            PF_STAMP(40);
             if (!PF_WAIT(B_APUB + buf, (c >> 1) & 1, 235)) return;
-            PF_STAMP(41);
             if (!PF_WAIT(B_QTFULL + buf, (c >> 1) & 1, 234)) return;
-            PF_STAMP(42);
             if (c >= 2 && !PF_WAIT(B_OFREE + buf, ((c >> 1) - 1) & 1, 233)) return;
-            PF_STAMP(43);
             tc_fence_after();
             gemm_ta<L_NSMN, 64, DK, 128>(t_o + buf * 64, t_a + buf * 64, smem_u32(smem + S_QT + buf * 16384));
             commit_uni(&bar[B_ODONE + buf]);
             commit_uni(&bar[B_QTEMPTY + buf]);
             commit_uni(&bar[B_S16FREE + buf]);
-            PF_STAMP(44);
         }
     } else {
         // ------------------------------------------------ ready flags in, consumed reports out -----------------
@@ -1041,12 +864,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
                     __nanosleep(200);
                 }
             }
-            PF_LAP_FLUSH(12);
         }
-    }
-    if (tim) {
-        atomicAdd(tim + 260 + (threadIdx.x >> 5), (unsigned long long)(clock64() - t_role));
-        atomicAdd(tim + 300 + (threadIdx.x >> 5), (unsigned long long)(globaltimer_ns() - t_ns));
     }
 }
 
@@ -1104,9 +922,6 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base_s;
-#ifdef PF_ENDS   // diagnostic builds: start and end of every CTA (globaltimer), words 0.. and 160.. of the timing block
-    if (tid == 0) ((unsigned long long*)(ws.status + 256))[blockIdx.x] = globaltimer_ns();
-#endif
 
     if (is_scan) scan_role(g, ws, S0, O, S_final, smem, bar, tb, (int)blockIdx.x);
     else flow_role<N>(maps, g, ws, beta, O, smem, bar, tb, (int)blockIdx.x - g.n_scan);
@@ -1114,9 +929,6 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
 
     tc_fence_before();
     __syncthreads();
-#ifdef PF_ENDS
-    if (tid == 0) ((unsigned long long*)(ws.status + 256))[160 + blockIdx.x] = globaltimer_ns();
-#endif
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
