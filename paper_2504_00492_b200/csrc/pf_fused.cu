@@ -18,10 +18,13 @@
 // rows of O that hold OI are updated by the scan a few chunk steps after the flow CTA wrote them, while they
 // are still in L2.  The only compulsory HBM traffic is one read of q, k, v, beta and one write of O.
 //
-// A flow CTA is software-pipelined over two chunks (15 warps):
-//   warps 0-3  "solve"  epilogue of G = K K^T (mask, column scaling, fp16) and the triangular inverse
-//   warps 4-7  "mid"    Uh half of [Uh | W], Xi^T half of [E | Xi^T] (into the ring), bf16 -> fp16 of V and K
-//   warps 8-11 "out"    W half, P^T, E half and [Qt^T | OI^T] (into the ring), bf16 -> fp16 of Q
+// A flow CTA is software-pipelined over two chunks (15 warps, two teams of workers):
+//   warps 0-3  "solve"  the chain that decides the period: epilogue of G = K K^T (mask, column scaling, fp16), the
+//                       16 x 16 diagonal blocks of the inverse (Neumann products on mma.sync, one warp per block)
+//                       and the recursive-doubling merges
+//   warps 4-11 "bulk"   one program for everything else, each step spread over all eight warps (two per lane
+//                       quarter of tensor memory): [Uh | W] into shared memory, P^T, bf16 -> fp16 of the next
+//                       chunk's V, K and Q, then the drains of E, Xi^T, Qt^T (into the ring) and OI (into O)
 //   warp 12             TMA loads (K and V double-buffered, Q single)
 //   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
 //   warp 14             ring back-pressure and ready flags
@@ -54,7 +57,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int FT = 480;                 // threads per CTA
+constexpr int FT = 512;                 // threads per CTA
 constexpr int DK = 128, DV = 128;
 
 // ---- ring slot layout (bytes) ---------------------------------------------------------------------------
@@ -90,7 +93,8 @@ constexpr int F_Q = 2 * F_REGION;               // 16 KB      Q
 constexpr int F_PT = F_Q + 16384;               // 16 KB      P^T
 constexpr int F_BETA = F_PT + 16384;            // 2 x 128 fp32
 constexpr int F_BAR = F_BETA + 1024;
-constexpr int SMEM_BYTES = F_BAR + 512;         // 230912
+constexpr int F_I16 = F_BAR + 512;              // 16 x 16 fp16 identity, unswizzled K-major (512 B)
+constexpr int SMEM_BYTES = F_I16 + 512;         // 231424
 // scan role
 constexpr int S_E = 0;                          // 2 x 32 KB  E images
 constexpr int S_XI = S_E + 2 * 32768;           // 2 x 32 KB  Xi images
@@ -105,28 +109,27 @@ enum {
     B_KFULL = 0,      // [2] TMA: K landed (bf16)
     B_VFULL = 2,      // [2]
     B_QFULL = 4,
-    B_K16 = 5,        // [2] mid: K converted to fp16
+    B_K16 = 5,        // [2] bulk: K converted to fp16
     B_V16 = 7,        // [2]
     B_Q16 = 9,
     B_GDONE = 10,     // mma: G complete
     B_GFREE = 11,     // solve: G drained from tensor memory
     B_XREADY = 12,    // [2] solve: X complete
     B_D2DONE = 14,    // mma: [Uh | W] complete
-    B_WUREADY = 15,   // mid: W, Uh in shared memory (RA drained)
+    B_WUREADY = 15,   // bulk: W, Uh in shared memory (RA drained)
     B_P0DONE = 16,    // mma: P0^T complete
-    B_PTREADY = 17,   // mid: P^T in shared memory (RC drained)
+    B_PTREADY = 17,   // bulk: P^T in shared memory (RC drained)
     B_D4DONE = 18,    // mma: [Qt^T | OI^T] complete (and everything issued before it)
+    B_D4FREE = 19,    // bulk: RC (Qt^T) and RD (OI^T) drained
+    B_RAFREE = 20,    // bulk: RA ([E | Xi^T]) drained
+    B_OUTDONE = 27,   // bulk: the chunk's images are stored
+    B_SLOTOK = 28,    // flag warp: the chunk's ring slot may be written
     B_RADONE = 29,    // mma: [E | Xi^T] complete
-    B_D4FREE = 19,    // out: RC (Qt^T) and RD (OI^T) drained
-    B_RAFREE = 20,    // out: RA drained
-    B_QCOPIED = 25,   // out: Q copied into registers
-    B_OUTDONE = 27,   // out: the chunk's images are stored
-    B_SLOTOK = 28,    // store warp: the chunk's ring slot may be written
     // scan role
     B_EFULL = 32,     // [2] producer: E image landed
     B_EEMPTY = 34,    // [2] chain: Delta of that chunk complete
     B_XIFULL = 36,    // [2] producer: Xi image landed
-    B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
+    B_XIEMPTY = 38,   // [2] mma: the Xi image has been read into its accumulator
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
     B_APUB = 44,      // [2 buffers] mma: Delta of the chunk complete (the O^T product may be issued)
@@ -139,11 +142,10 @@ enum {
 
 #define PF_WAIT(idx, parity, code) mbar_wait_clk(&bar[idx], (uint32_t)(parity), err, code)
 
-// byte offset of the 16-byte chunk `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
-__device__ __forceinline__ uint32_t chunk_off(int row, int col8, int R) {
-    return (uint32_t)(col8 >> 3) * (uint32_t)R * 128u + (uint32_t)row * 128u + ((((uint32_t)col8 & 7u) ^ ((uint32_t)row & 7u)) << 4);
+__device__ __forceinline__ uint4 pack8n(const uint32_t* r) {
+    return make_uint4(pack_h2(__uint_as_float(r[0]), __uint_as_float(r[1])), pack_h2(__uint_as_float(r[2]), __uint_as_float(r[3])),
+                      pack_h2(__uint_as_float(r[4]), __uint_as_float(r[5])), pack_h2(__uint_as_float(r[6]), __uint_as_float(r[7])));
 }
-
 __device__ __forceinline__ uint4 pack8(const uint32_t* r, float scale) {
     return make_uint4(pack_h2(__uint_as_float(r[0]) * scale, __uint_as_float(r[1]) * scale),
                       pack_h2(__uint_as_float(r[2]) * scale, __uint_as_float(r[3]) * scale),
@@ -151,12 +153,12 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* r, float scale) {
                       pack_h2(__uint_as_float(r[6]) * scale, __uint_as_float(r[7]) * scale));
 }
 
-// bf16 -> fp16 in place, elementwise (so the swizzled layout is untouched); 128 threads
-static __device__ __noinline__ void cvt_region(uint8_t* base, int bytes, int t128) {
+// bf16 -> fp16 in place, elementwise (so the swizzled layout is untouched); `nthr` threads, this one is `t`
+static __device__ __noinline__ void cvt_region(uint8_t* base, int bytes, int t, int nthr) {
     uint4* p = (uint4*)base;
     const int chunks = bytes >> 4;
 #pragma unroll 4
-    for (int e = t128; e < chunks; e += 128) {
+    for (int e = t; e < chunks; e += nthr) {
         uint4 val = p[e];
         uint32_t* w = (uint32_t*)&val;
 #pragma unroll
@@ -166,75 +168,6 @@ static __device__ __noinline__ void cvt_region(uint8_t* base, int bytes, int t12
         }
         p[e] = val;
     }
-}
-
-// One level of the recursive-doubling inverse (Proposition on block-triangular inversion): diagonal blocks of
-// size S are merged into blocks of size 2S,  X_hi,lo = -X_hi,hi A_hi,lo X_lo,lo.  Task = (merge, 16-row
-// strip): N/32 tasks, one warp each; the four solve warps synchronise on named barrier 1.
-template <int N, int S>
-__device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, int lane) {
-    constexpr int TASKS = N / 32;
-    constexpr int STRIPS = S / 16;
-    constexpr int NT = S / 8;
-    float z[NT][4];
-    const bool has_task = warp < TASKS;
-    const int q = warp / STRIPS, strip = warp % STRIPS;
-    const int lo0 = 2 * S * q, hi0 = lo0 + S, R0 = hi0 + 16 * strip;
-    const int id = lane >> 3;
-    if (has_task) {
-        float u[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) u[nt][e] = 0.f;
-        // (all column offsets below are multiples of 8, all row offsets multiples of 8 plus a lane term)
-        const int a_row = R0 + (lane & 15), a_c8 = (hi0 >> 3) + (lane >> 4);
-        const int b_rowl = (lane & 7) + ((id & 1) << 3), b_c8l = (id >> 1);
-#pragma unroll
-        for (int kk = 0; kk < S / 16; ++kk) {
-            if (kk > strip) continue;   // X_hi,hi is lower triangular
-            uint32_t a[4];
-            ldmatrix_x4(a, xb + chunk_off(a_row, a_c8 + 2 * kk, N));
-#pragma unroll
-            for (int np = 0; np < S / 16; ++np) {
-                uint32_t b[4];
-                ldmatrix_x4_trans(b, xb + chunk_off(hi0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
-                mma_16816(u[2 * np], a, b[0], b[1]);
-                mma_16816(u[2 * np + 1], a, b[2], b[3]);
-            }
-        }
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) z[nt][e] = 0.f;
-#pragma unroll
-        for (int kk = 0; kk < S / 16; ++kk) {
-            uint32_t a[4];
-            a[0] = pack_h2(u[2 * kk][0], u[2 * kk][1]);
-            a[1] = pack_h2(u[2 * kk][2], u[2 * kk][3]);
-            a[2] = pack_h2(u[2 * kk + 1][0], u[2 * kk + 1][1]);
-            a[3] = pack_h2(u[2 * kk + 1][2], u[2 * kk + 1][3]);
-#pragma unroll
-            for (int np = 0; np < S / 16; ++np) {
-                if (np > kk) continue;  // X_lo,lo is lower triangular
-                uint32_t b[4];
-                ldmatrix_x4_trans(b, xb + chunk_off(lo0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
-                mma_16816(z[2 * np], a, b[0], b[1]);
-                mma_16816(z[2 * np + 1], a, b[2], b[3]);
-            }
-        }
-    }
-    named_bar(1, 128);   // every strip has read A_hi,lo before anyone overwrites it
-    if (has_task) {
-        const int gq = lane >> 2, t4 = lane & 3;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int c8 = (lo0 >> 3) + nt;
-            *(uint32_t*)(xg + chunk_off(R0 + gq, c8, N) + 4 * t4) = pack_h2(-z[nt][0], -z[nt][1]);
-            *(uint32_t*)(xg + chunk_off(R0 + gq + 8, c8, N) + 4 * t4) = pack_h2(-z[nt][2], -z[nt][3]);
-        }
-    }
-    named_bar(1, 128);
 }
 
 // =============================================================================================================
@@ -250,8 +183,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
     const int nk = fid < g.items ? (g.items - fid + g.n_flow - 1) / g.n_flow : 0;
     const uint32_t RA = tb, RG = tb + 256, RC = tb + 384, RD = tb + 448;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    constexpr uint32_t KV_SLAB = N * 128;                 // bytes of one 64-column slab of K / V / W / Uh
-    constexpr uint32_t K_BYTES = N * 256;
     constexpr int X_OFF = 0, V_OFF = N * 256, K_OFF = 2 * N * 256;   // inside a parity region
 
     auto item = [&](int k, int& seq, int& c) {
@@ -264,6 +195,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
         // ------------------------------------------------ solve: G epilogue + triangular inverse -------------
         const int m = tid;
         const int row_lim = (m / g.rm) * g.rm; // rows m' < row_lim: earlier tokens (sum form) / earlier rows (product form)
+        const bool deep = g.rm == 1;           // (with groups of two or more rows the 16 x 16 blocks have A^8 = 0)
         float* sBeta = (float*)(smem + F_BETA);
         float beta_next = 0.f;
         if (nk > 0) {
@@ -271,9 +203,9 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             item(0, seq, c);
             const int nv = min(C, g.L - c * C) * r;
             if (m < nv) {
-                    const long long bi = ((long long)seq * g.L + (long long)c * C) * r + m;
-                    beta_next = g.b32 ? g.b32[bi] : __bfloat162float(beta[bi]);
-                }
+                const long long bi = ((long long)seq * g.L + (long long)c * C) * r + m;
+                beta_next = g.b32 ? g.b32[bi] : __bfloat162float(beta[bi]);
+            }
         }
 #pragma unroll 1
         for (int k = 0; k < nk; ++k) {
@@ -295,361 +227,360 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
             bool ok = true;
-            if (k >= 2) ok = PF_WAIT(B_D4DONE, (k - 2) & 1, 101);     // W of chunk k-2 (in this X region) has been read
+            // (G of chunk k is issued only once W of chunk k-2, in this X region, has been read by all of that chunk's products)
             sB[m] = bm;     // (the beta half of chunk k-2 was last read by that chunk's [Uh | W] epilogue)
-            ok = ok && PF_WAIT(B_GDONE, k & 1, 102);
+            ok = PF_WAIT(B_GDONE, k & 1, 102);
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
-            // A = Mstrict (.) (G diag(beta)) as fp16 into X; column groups right of the warp's rows are zero
+            // A = Mstrict (.) (G diag(beta)) as fp16 into X.  Warp w holds rows 32w .. 32w+31: the 32-column groups
+            // left of 32w lie entirely below the mask's edge, the group at 32w holds the edge, the groups to the
+            // right are zero.
+            if (32 * warp < N) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < N; c0 += 32) {
-                uint32_t rr[32];
-                const bool live = c0 < 32 * (warp + 1);
-                if (live) {
-                    tmem_ld32(RG + lane_base + c0, rr);
-                    tmem_ld_wait();
-                }
-                if (m < N) {
+                for (int c0 = 0; c0 < N; c0 += 32) {
+                    if (c0 > 32 * warp) {
 #pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8) {
-                        uint4 pk = make_uint4(0, 0, 0, 0);
-                        if (live) {
-                            const float4 b0 = *(const float4*)(sB + c0 + j8), b1 = *(const float4*)(sB + c0 + j8 + 4);
-                            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(sX + chunk_off(m, (c0 >> 3) + j8, N)) = make_uint4(0, 0, 0, 0);
+                        continue;
+                    }
+                    uint32_t rr[32];
+                    tmem_ld32(RG + lane_base + c0, rr);
+                    float bb[32];
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 bv = *(const float4*)(sB + c0 + 4 * j4);
+                        bb[4 * j4] = bv.x; bb[4 * j4 + 1] = bv.y; bb[4 * j4 + 2] = bv.z; bb[4 * j4 + 3] = bv.w;
+                    }
+                    tmem_ld_wait();
+                    if (c0 < 32 * warp) {
+#pragma unroll
+                        for (int j8 = 0; j8 < 32; j8 += 8) {
                             float a[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) a[j] = (c0 + j8 + j < row_lim) ? bb[j] * __uint_as_float(rr[j8 + j]) : 0.f;
-                            pk = make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
+                            for (int j = 0; j < 8; ++j) a[j] = bb[j8 + j] * __uint_as_float(rr[j8 + j]);
+                            *(uint4*)(sX + chunk_off(m, (c0 + j8) >> 3, N)) =
+                                make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                         }
-                        *(uint4*)(sX + chunk_off(m, (c0 + j8) >> 3, N)) = pk;
+                    } else {
+#pragma unroll
+                        for (int j8 = 0; j8 < 32; j8 += 8) {
+                            float a[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) a[j] = (c0 + j8 + j < row_lim) ? bb[j8 + j] * __uint_as_float(rr[j8 + j]) : 0.f;
+                            *(uint4*)(sX + chunk_off(m, (c0 + j8) >> 3, N)) =
+                                make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
+                        }
                     }
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_GFREE]);
-            named_bar(1, 128);
-            // 16x16 diagonal blocks: forward substitution, one thread per column of one block (fp32)
-            float x[16];
-            const int bk = tid >> 4, cc = tid & 15;
-            if (tid < N) {
-                const uint8_t* blk = sX + (bk >> 2) * (N * 128) + (16 * bk) * 128;    // row 16*bk of the block's slab
-                const int c8 = (2 * bk) & 7;                                          // first 16-byte chunk of the block
-#pragma unroll
-                for (int mm = 0; mm < 16; ++mm) {
-                    const uint4 lo = *(const uint4*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4));
-                    const uint4 hi = *(const uint4*)(blk + mm * 128 + (((c8 + 1) ^ (mm & 7)) << 4));
-                    const __half2* hl = (const __half2*)&lo;
-                    const __half2* hh = (const __half2*)&hi;
-                    float a[16];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 f0 = __half22float2(hl[e]), f1 = __half22float2(hh[e]);
-                        a[2 * e] = f0.x; a[2 * e + 1] = f0.y; a[8 + 2 * e] = f1.x; a[9 + 2 * e] = f1.y;
-                    }
-                    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-                    for (int mp = 0; mp < mm; ++mp) {
-                        if (mp & 1) acc1 = fmaf(a[mp], x[mp], acc1);
-                        else acc0 = fmaf(a[mp], x[mp], acc0);
-                    }
-                    x[mm] = ((mm == cc) ? 1.f : 0.f) - (acc0 + acc1);
-                }
+            // 16 x 16 diagonal blocks 2w and 2w+1: their rows were written by this warp
+            __syncwarp();
+            if (32 * warp < N) {
+                diag_inverse16(x_b, sX, 2 * warp, lane, N, deep);
+                diag_inverse16(x_b, sX, 2 * warp + 1, lane, N, deep);
             }
             named_bar(1, 128);
-            if (tid < N) {
-                uint8_t* blk = sX + (bk >> 2) * (N * 128) + (16 * bk) * 128;
-                const int c8 = ((2 * bk) & 7) + (cc >> 3);
-#pragma unroll
-                for (int mm = 0; mm < 16; ++mm)
-                    *(__half*)(blk + mm * 128 + ((c8 ^ (mm & 7)) << 4) + (cc & 7) * 2) = __float2half_rn(x[mm]);
-            }
-            named_bar(1, 128);
-            merge_level<N, 16>(x_b, sX, warp, lane);
-            merge_level<N, 32>(x_b, sX, warp, lane);
-            if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
+            merge_level<N, 16, 1>(x_b, sX, warp, lane);
+            merge_level<N, 32, 1>(x_b, sX, warp, lane);
+            if (N == 128) merge_level<N, 64, 1>(x_b, sX, warp, lane);
             fence_async_smem();
             mbar_arrive(&bar[B_XREADY + b]);
         }
-    } else if (warp < 8) {
-        // ------------------------------------------------ mid: Uh and Xi^T halves, conversions of V and K -----
-        const int m = tid - 128;
-        const float* sBeta = (const float*)(smem + F_BETA);
-        if (nk > 0) {
-            if (!PF_WAIT(B_VFULL + 0, 0, 112)) return;
-            cvt_region(smem + V_OFF, K_BYTES, m);
-            fence_async_smem();
-            mbar_arrive(&bar[B_V16 + 0]);
-            // (K only once its Gram product has read the bf16 tile)
-            if (!PF_WAIT(B_KFULL + 0, 0, 111) || !PF_WAIT(B_GDONE, 0, 110)) return;
-            cvt_region(smem + K_OFF, K_BYTES, m);
-            fence_async_smem();
-            mbar_arrive(&bar[B_K16 + 0]);
-        }
-#pragma unroll 1
-        for (int k = 0; k < nk; ++k) {
-            const int b = k & 1, b1 = b ^ 1;
-            int seq, c;
-            item(k, seq, c);
-            uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
-            // ---- RA = X [V | K], first half:  Uh = diag(beta) (X V), fp16, over V
-            if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
-            tc_fence_after();
-            {
-                const float bm = (m < N) ? sBeta[b * 128 + m] : 0.f;
-                uint8_t* sU = smem + b * F_REGION + V_OFF;
-#pragma unroll 1
-                for (int c0 = 0; c0 < DV; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RA + lane_base + c0, rr);
-                    tmem_ld_wait();
-                    if (m < N) {
-#pragma unroll
-                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(sU + chunk_off(m, (c0 >> 3) + j8, N)) = pack8(rr + 8 * j8, bm);
-                    }
-                }
-            }
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive(&bar[B_WUREADY]);
-            // ---- conversions for chunk k+1
-            if (k + 1 < nk) {
-                if (!PF_WAIT(B_VFULL + b1, ((k + 1) >> 1) & 1, 115)) return;
-                cvt_region(smem + b1 * F_REGION + V_OFF, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_V16 + b1]);
-                if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 113) || !PF_WAIT(B_GDONE, (k + 1) & 1, 119)) return;
-                cvt_region(smem + b1 * F_REGION + K_OFF, K_BYTES, m);
-                fence_async_smem();
-                mbar_arrive(&bar[B_K16 + b1]);
-            }
-            // ---- RA = [E | Xi^T], second half: row j = m of Xi^T, one 16-byte piece per column group, into the ring
-            if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
-            tc_fence_after();
-            {
-                uint8_t* xrow = slot + SLOT_XI + m * 16;
-#pragma unroll 1
-                for (int c0 = 0; c0 < DK; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RA + lane_base + DK + c0, rr);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(xrow + ((c0 >> 3) + j8) * 2048) = pack8(rr + 8 * j8, 1.f);
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(&bar[B_RAFREE]);
-            mbar_arrive(&bar[B_OUTDONE]);
-        }
     } else if (warp < 12) {
-        // ------------------------------------------------ out: W half, P^T, E / Qt / OI into the ring, Q ---------
-        const int i = tid - 256;
-        const int tokm = i / r;
+        // ------------------------------------------------ bulk: everything else, eight warps per step ----------
+        // thread (h, m): lane quarter of row m = 32 (warp & 3) + lane; h = 0 takes the Uh / Xi^T / OI side of
+        // every step, h = 1 the W / E / Qt side.
+        //
+        // Thread 0 of the team also issues the TMA loads, each right after the wait that shows its buffer free.
+        const int bt = tid - 128;
+        const int h = bt >> 7, m = bt & 127;
+        const int tokm = m / r;
         const float* sBeta = (const float*)(smem + F_BETA);
-        uint8_t* sPT = smem + F_PT;
-        const uint8_t* sQ = smem + F_Q;
-        uint32_t qreg[32];      // column i of Q (fp16 pairs over t): lets the Q buffer take the next chunk early
-        auto q_prepare = [&](int k) -> bool {
-            // (a failed wait must not strand the others at the barrier: the barrier carries the outcome)
-            bool okq = PF_WAIT(B_QFULL, k & 1, 114);
-            if (okq) cvt_region(smem + F_Q, 16384, i);
+        const uint32_t sw16 = (uint32_t)(m & 7) << 4;
+        constexpr uint32_t KV_SLAB = N * 128;                 // bytes of one 64-column slab of K / V / W / Uh
+        constexpr uint32_t K_BYTES = N * 256;
+        const int dq_c = g.n_flow / nseq, dq_s = g.n_flow - dq_c * nseq;            // how (chunk, sequence) advance per item
+        auto advance = [&](int& sq, int& ch) {
+            sq += dq_s;
+            ch += dq_c;
+            if (sq >= nseq) { sq -= nseq; ++ch; }
+        };
+        auto load_k = [&](int bb, int sq, int ch) {
+            mbar_expect_tx(&bar[B_KFULL + bb], K_BYTES);
+            for (int hh = 0; hh < 2; ++hh)
+                tma_load_3d(smem + bb * F_REGION + K_OFF + hh * KV_SLAB, &maps.k, 64 * hh, ch * C * r, sq, &bar[B_KFULL + bb]);
+        };
+        auto load_v = [&](int bb, int sq, int ch) {
+            mbar_expect_tx(&bar[B_VFULL + bb], K_BYTES);
+            for (int hh = 0; hh < 2; ++hh)
+                tma_load_3d(smem + bb * F_REGION + V_OFF + hh * KV_SLAB, &maps.v, 64 * hh, ch * C * r, sq, &bar[B_VFULL + bb]);
+        };
+        auto load_q = [&](int sq, int ch) {
+            mbar_expect_tx(&bar[B_QFULL], (uint32_t)C * 256);
+            for (int hh = 0; hh < 2; ++hh) tma_load_3d(smem + F_Q + hh * 8192, &maps.q, 64 * hh, ch * C, sq, &bar[B_QFULL]);
+        };
+        // conversions of chunk kk's V and K tiles (buffers kk & 1); K only once its Gram product has read the bf16 tile
+        auto convert_vk = [&](int kk) -> bool {
+            const int bb = kk & 1, ph = (kk >> 1) & 1;
+            if (!PF_WAIT(B_VFULL + bb, ph, 112)) return false;
+            cvt_region(smem + bb * F_REGION + V_OFF, K_BYTES, bt, 256);
             fence_async_smem();
-            if (okq) mbar_arrive(&bar[B_Q16]);
-            if (!named_bar_and(3, 128, okq)) return false;
-            const uint8_t* qcol = sQ + (i >> 6) * 8192 + (i & 7) * 2;
-            const int ci = (i & 63) >> 3;
-#pragma unroll
-            for (int t = 0; t < 64; t += 2) {
-                const uint32_t lo = *(const uint16_t*)(qcol + t * 128 + ((ci ^ (t & 7)) << 4));
-                const uint32_t hi = *(const uint16_t*)(qcol + (t + 1) * 128 + ((ci ^ ((t + 1) & 7)) << 4));
-                qreg[t >> 1] = lo | (hi << 16);
-            }
-            mbar_arrive(&bar[B_QCOPIED]);
+            mbar_arrive(&bar[B_V16 + bb]);
+            if (!PF_WAIT(B_KFULL + bb, ph, 111) || !PF_WAIT(B_GDONE, kk & 1, 110)) return false;
+            cvt_region(smem + bb * F_REGION + K_OFF, K_BYTES, bt, 256);
+            fence_async_smem();
+            mbar_arrive(&bar[B_K16 + bb]);
             return true;
         };
-        if (nk > 0 && !q_prepare(0)) return;
+        auto convert_q = [&](int kk) -> bool {
+            if (!PF_WAIT(B_QFULL, kk & 1, 114)) return false;
+            cvt_region(smem + F_Q, 16384, bt, 256);
+            fence_async_smem();
+            mbar_arrive(&bar[B_Q16]);
+            return true;
+        };
+        int seq, c;
+        item(0, seq, c);
+        if (nk > 0) {
+            if (bt == 0) {
+                int s1 = seq, c1 = c;
+                load_k(0, seq, c);
+                load_q(seq, c);
+                load_v(0, seq, c);
+                if (nk > 1) {
+                    advance(s1, c1);
+                    load_k(1, s1, c1);
+                    load_v(1, s1, c1);
+                }
+            }
+            if (!convert_vk(0) || !convert_q(0)) return;
+        }
 #pragma unroll 1
         for (int k = 0; k < nk; ++k) {
             const int b = k & 1;
-            int seq, c;
-            item(k, seq, c);
             const int Cv = min(C, g.L - c * C), nv = Cv * r;
             uint8_t* slot = ws.ring + ((size_t)seq * g.R + (c % g.R)) * SLOT_BYTES;
-            // ---- RA = X [V | K], second half:  -W = -diag(beta) (X K), fp16, over X
-            if (!PF_WAIT(B_D2DONE, k & 1, 125)) return;
+            // ---- RA = X [V | K]:  h = 0: Uh = diag(beta) (X V) over V;  h = 1: -W = -diag(beta) (X K) over X   (fp16)
+            if (!PF_WAIT(B_D2DONE, k & 1, 118)) return;
             tc_fence_after();
             {
-                const float bm = (i < N) ? -sBeta[b * 128 + i] : 0.f;
-                uint8_t* sW = smem + b * F_REGION + X_OFF;
+                const float bs = (m < N) ? sBeta[b * 128 + m] : 0.f;
+                const float bm = h ? -bs : bs;
+                uint8_t* mrow = smem + b * F_REGION + (h ? X_OFF : V_OFF) + m * 128;
+                const uint32_t src = RA + lane_base + h * 128;
 #pragma unroll 1
-                for (int c0 = 0; c0 < DK; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RA + lane_base + DV + c0, rr);
-                    tmem_ld_wait();
-                    if (i < N) {
+                for (int sl = 0; sl < 2; ++sl) {                 // 64-column slab
 #pragma unroll
-                        for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(sW + chunk_off(i, (c0 >> 3) + j8, N)) = pack8(rr + 8 * j8, bm);
+                    for (int st4 = 0; st4 < 4; ++st4) {          // 16 columns = two 16-byte pieces
+                        uint32_t rr[16];
+                        tmem_ld16(src + 64 * sl + 16 * st4, rr);
+                        tmem_ld_wait();
+                        if (m < N) {
+                            *(uint4*)(mrow + sl * (N * 128) + (((uint32_t)(2 * st4) << 4) ^ sw16)) = pack8(rr, bm);
+                            *(uint4*)(mrow + sl * (N * 128) + (((uint32_t)(2 * st4 + 1) << 4) ^ sw16)) = pack8(rr + 8, bm);
+                        }
                     }
                 }
             }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_WUREADY]);
-            // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]   (P^T of chunk k-1 was last read by its MMA4)
-            if (k >= 1 && !PF_WAIT(B_D4DONE, (k - 1) & 1, 116)) return;
+            // ---- P^T = P0^T (.) Mincl as fp16 [m rows][64 t]: 32 columns per half  (P^T of chunk k-1 was last read by
+            //      that chunk's Qt / OI products, complete before the drains of chunk k-1 started)
             if (!PF_WAIT(B_P0DONE, k & 1, 117)) return;
             tc_fence_after();
-#pragma unroll 1
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(RC + lane_base + c0, rr);
-                tmem_ld_wait();
-                if (i < N) {
+            {
+                const int lo = m < nv ? tokm : 64;               // tokens t in [lo, Cv) see row m
+                uint8_t* prow_ = smem + F_PT + m * 128;          // (one slab: 64 columns)
 #pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8) {
-                        float a[8];
+                for (int st2 = 0; st2 < 2; ++st2) {
+                    const int c0 = 32 * h + 16 * st2;
+                    uint32_t rr[16];
+                    tmem_ld16(RC + lane_base + c0, rr);
+                    tmem_ld_wait();
+                    if (m < N) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int t = c0 + j8 + j;
-                            a[j] = (tokm <= t && t < Cv && i < nv) ? __uint_as_float(rr[j8 + j]) : 0.f;
+                        for (int j8 = 0; j8 < 16; j8 += 8) {
+                            float a[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int t = c0 + j8 + j;
+                                a[j] = (t >= lo && t < Cv) ? __uint_as_float(rr[j8 + j]) : 0.f;
+                            }
+                            *(uint4*)(prow_ + (((uint32_t)((c0 + j8) >> 3) << 4) ^ sw16)) =
+                                make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                         }
-                        *(uint4*)(sPT + chunk_off(i, (c0 + j8) >> 3, N)) =
-                            make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                     }
                 }
             }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_PTREADY]);
-            // ---- RA = [E | Xi^T], first half: row i of E, one 16-byte piece per column group, into the ring
-            if (!PF_WAIT(B_SLOTOK, k & 1, 121) || !PF_WAIT(B_RADONE, k & 1, 123)) return;
+            // ---- conversions for chunk k+1 (while [E | Xi^T] of chunk k is formed)
+            if (k + 1 < nk && !convert_vk(k + 1)) return;
+            // ---- RA = [E | Xi^T]: h = 1: row m of E, h = 0: row m of Xi^T, one 16-byte piece per column group, into the ring
+            if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
             tc_fence_after();
             {
-                uint8_t* erow = slot + SLOT_E + i * 16;
+                uint8_t* row = slot + (h ? SLOT_E : SLOT_XI) + m * 16;
+                const uint32_t src = RA + lane_base + (h ? 0 : DK);
 #pragma unroll 1
-                for (int c0 = 0; c0 < DK; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RA + lane_base + c0, rr);
-                    tmem_ld_wait();
+                for (int sl = 0; sl < 2; ++sl) {
 #pragma unroll
-                    for (int j8 = 0; j8 < 4; ++j8) *(uint4*)(erow + ((c0 >> 3) + j8) * 2048) = pack8(rr + 8 * j8, 1.f);
+                    for (int st4 = 0; st4 < 4; ++st4) {
+                        uint32_t rr[16];
+                        tmem_ld16(src + 64 * sl + 16 * st4, rr);
+                        tmem_ld_wait();
+                        *(uint4*)(row + sl * 16384 + (2 * st4) * 2048) = pack8n(rr);
+                        *(uint4*)(row + sl * 16384 + (2 * st4 + 1) * 2048) = pack8n(rr + 8);
+                    }
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
-            // ---- RC: Qt^T[i][t] = Q[t][i] - (W^T P^T)[i][t] (row i of the Qt image);  RD: OI^T[j][t] -> OI[t][j] (fp32)
+            // ---- K of chunk k+2 into the buffer that [E | Xi^T] of this chunk has just finished reading
+            if (bt == 0 && k + 2 < nk) {
+                int s2 = seq, c2 = c;
+                advance(s2, c2);
+                advance(s2, c2);
+                load_k(b, s2, c2);
+            }
+            // ---- h = 1: RC: Qt^T (row i = m of the Qt image);  h = 0: RD: OI^T[j][t] -> OI[t][j = m] (fp32) into the rows of O
             if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
             tc_fence_after();
-            {
-                uint8_t* qrow = slot + SLOT_QT + i * 16;
-#pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RC + lane_base + c0, rr);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j8 = 0; j8 < 4; ++j8) {
-                        uint32_t w4[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t qq = qreg[(c0 >> 1) + 4 * j8 + j];
-                            const float2 qf = __half22float2(*reinterpret_cast<const __half2*>(&qq));
-                            w4[j] = pack_h2(__uint_as_float(rr[8 * j8 + 2 * j]) + qf.x, __uint_as_float(rr[8 * j8 + 2 * j + 1]) + qf.y);
-                        }
-                        *(uint4*)(qrow + ((c0 >> 3) + j8) * 2048) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-                    }
+            if (bt == 0 && k + 1 < nk) {       // (the Q tile and Uh of this chunk have been read by its last product)
+                int s2 = seq, c2 = c;
+                advance(s2, c2);
+                load_q(s2, c2);
+                if (k + 2 < nk) {
+                    advance(s2, c2);
+                    load_v(b, s2, c2);
                 }
-                float* oi = O + ((long long)seq * g.L + (long long)c * C) * DV + i;     // OI[t][j = i] into the rows of O
-#pragma unroll 1
-                for (int c0 = 0; c0 < 64; c0 += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(RD + lane_base + c0, rr);
-                    tmem_ld_wait();
-                    const int lim = Cv - c0;
+            }
+            if (h == 1) {
+                uint8_t* qrow = slot + SLOT_QT + m * 16;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (j < lim) oi[(c0 + j) * DV] = __uint_as_float(rr[j]);
+                for (int st4 = 0; st4 < 4; ++st4) {
+                    uint32_t rr[16];
+                    tmem_ld16(RC + lane_base + 16 * st4, rr);
+                    tmem_ld_wait();
+                    *(uint4*)(qrow + (2 * st4) * 2048) = pack8n(rr);
+                    *(uint4*)(qrow + (2 * st4 + 1) * 2048) = pack8n(rr + 8);
+                }
+            } else {
+                float* oi = O + ((long long)seq * g.L + (long long)c * C) * DV + m;
+                if (Cv == 64) {
+#pragma unroll
+                    for (int st4 = 0; st4 < 4; ++st4) {
+                        uint32_t rr[16];
+                        tmem_ld16(RD + lane_base + 16 * st4, rr);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) oi[(16 * st4 + j) * DV] = __uint_as_float(rr[j]);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                        uint32_t rr[16];
+                        tmem_ld16(RD + lane_base + c0, rr);
+                        tmem_ld_wait();
+                        const int lim = Cv - c0;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (j < lim) oi[(c0 + j) * DV] = __uint_as_float(rr[j]);
+                    }
                 }
             }
             tc_fence_before();
             mbar_arrive(&bar[B_D4FREE]);
             mbar_arrive(&bar[B_OUTDONE]);
-            // ---- Q of the next chunk: convert in place, then take this thread's column
-            if (k + 1 < nk && !q_prepare(k + 1)) return;
-        }
-    } else if (warp == 12) {
-        // ------------------------------------------------ TMA loads -------------------------------------------
-        if (lane == 0) {
-#pragma unroll 1
-            for (int j = 0; j < nk; ++j) {
-                const int b = j & 1;
-                int seq, c;
-                item(j, seq, c);
-                // K and V: their regions were last read by the MMAs of chunk j-2
-                if (j >= 2 && !PF_WAIT(B_D4DONE, (j - 2) & 1, 131)) return;
-                mbar_expect_tx(&bar[B_KFULL + b], K_BYTES);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_3d(smem + b * F_REGION + K_OFF + h * KV_SLAB, &maps.k, 64 * h, c * C * r, seq, &bar[B_KFULL + b]);
-                // Q: single buffer, free once P0^T of chunk j-1 is complete and the out warps hold their copy
-                if (j >= 1 && (!PF_WAIT(B_P0DONE, (j - 1) & 1, 132) || !PF_WAIT(B_QCOPIED, (j - 1) & 1, 136))) return;
-                mbar_expect_tx(&bar[B_QFULL], (uint32_t)C * 256);
-                for (int h = 0; h < 2; ++h) tma_load_3d(smem + F_Q + h * 8192, &maps.q, 64 * h, c * C, seq, &bar[B_QFULL]);
-                mbar_expect_tx(&bar[B_VFULL + b], K_BYTES);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_3d(smem + b * F_REGION + V_OFF + h * KV_SLAB, &maps.v, 64 * h, c * C * r, seq, &bar[B_VFULL + b]);
-            }
+            // ---- Q of chunk k+1
+            if (k + 1 < nk && !convert_q(k + 1)) return;
+            advance(seq, c);
         }
     } else if (warp == 13) {
-        // ------------------------------------------------ MMA issue (whole warp, converged) --------------------
-        if (nk > 0) {
-            const uint32_t q_b = smem_u32(smem + F_Q), pt_b = smem_u32(smem + F_PT);
-            if (!PF_WAIT(B_KFULL + 0, 0, 141)) return;
-            tc_fence_after();
-            {
-                const uint32_t k_b = smem_u32(smem + K_OFF);
-                gemm_uni<false, false, N, DK, N, N, true>(RG, k_b, k_b);     // G(0) = K K^T from the bf16 tile
-                commit_uni(&bar[B_GDONE]);
-            }
+        // ------------------------------------------------ MMA issue, first of three warps: G and [Uh | W] --------
+        // Five products per chunk -- G, P0^T, [Uh | W], [E | Xi^T], [Qt^T | OI^T] -- are issued by three warps on three
+        // different schedulers (an issuing warp shares its scheduler with busy worker warps, and one warp alone cannot
+        // issue fast enough to keep the tensor pipe fed).  Each product is issued as soon as its inputs are there and
+        // its accumulator is free, in chunk order per product; this warp polls for whichever of its two is ready, so
+        // that G of the next chunk (which the solve warps wait for) is never held back by X of this one, or vice versa.
+        int ig = 0, ip3 = 0;
+        const uint32_t reg0 = smem_u32(smem);
+        auto ph2 = [](int kk) { return (uint32_t)((kk >> 1) & 1); };
+        long long t_last = clock64();
 #pragma unroll 1
-            for (int k = 0; k < nk; ++k) {
-                const int b = k & 1, b1 = b ^ 1;
-                const uint32_t x_b = smem_u32(smem + b * F_REGION + X_OFF), v_b = x_b + V_OFF, k_b = x_b + K_OFF;
-                // [Uh | W] (before the row scaling) = X [V | K]
-                if (!PF_WAIT(B_XREADY + b, (k >> 1) & 1, 142) || !PF_WAIT(B_V16 + b, (k >> 1) & 1, 143) ||
-                    !PF_WAIT(B_K16 + b, (k >> 1) & 1, 140))
-                    return;
-                if (k >= 1 && !PF_WAIT(B_RAFREE, (k - 1) & 1, 144)) return;
+        while (ip3 < nk) {
+            bool progress = false;
+            // (G of chunk ig: its K tile has landed; the solve warps have drained G of chunk ig-1; the bulk warps have all seen
+            //  G of chunk ig-1 complete -- they convert that chunk's K only then -- so that nobody can miss a phase of the
+            //  barrier G completes on; and the last product of chunk ig-2 is done with W in the X region G's epilogue goes to)
+            if (ig < nk && mbar_test(&bar[B_KFULL + (ig & 1)], ph2(ig)) &&
+                (ig == 0 || (mbar_test(&bar[B_GFREE], (ig - 1) & 1) && mbar_test(&bar[B_K16 + ((ig - 1) & 1)], ph2(ig - 1)))) &&
+                (ig < 2 || mbar_test(&bar[B_D4DONE], (ig - 2) & 1))) {
                 tc_fence_after();
-                gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, v_b);
+                const uint32_t k_b = reg0 + (ig & 1) * F_REGION + K_OFF;
+                gemm_uni<false, false, N, DK, N, N, true>(RG, k_b, k_b);            // G = K K^T from the bf16 tile as it landed
+                commit_uni(&bar[B_GDONE]);
+                ++ig;
+                progress = true;
+            }
+            if (mbar_test(&bar[B_XREADY + (ip3 & 1)], ph2(ip3)) && mbar_test(&bar[B_V16 + (ip3 & 1)], ph2(ip3)) &&
+                mbar_test(&bar[B_K16 + (ip3 & 1)], ph2(ip3)) && (ip3 == 0 || mbar_test(&bar[B_RAFREE], (ip3 - 1) & 1))) {
+                tc_fence_after();
+                const uint32_t x_b = reg0 + (ip3 & 1) * F_REGION + X_OFF;
+                gemm_uni<false, true, DV + DK, N, N, N>(RA, x_b, x_b + V_OFF);      // [Uh | W] (before the row scaling) = X [V | K]
                 commit_uni(&bar[B_D2DONE]);
-                // G of the next chunk, from its bf16 tile (RG: the solve warps have drained G of this chunk)
-                if (k + 1 < nk) {
-                    if (!PF_WAIT(B_KFULL + b1, ((k + 1) >> 1) & 1, 145) || !PF_WAIT(B_GFREE, k & 1, 146)) return;
-                    tc_fence_after();
-                    const uint32_t k1_b = smem_u32(smem + b1 * F_REGION + K_OFF);
-                    gemm_uni<false, false, N, DK, N, N, true>(RG, k1_b, k1_b);
-                    commit_uni(&bar[B_GDONE]);
-                }
-                // P0^T = K Q^T   (RC and RD: Qt^T and OI^T of chunk k-1 have been drained)
-                if (!PF_WAIT(B_Q16, k & 1, 148)) return;
-                if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
-                tc_fence_after();
-                gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
-                commit_uni(&bar[B_P0DONE]);
-                // E = K^T (-W)  (lanes i, columns i'),   Xi^T = Uh^T K  (lanes j, columns i)
-                if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
-                tc_fence_after();
-                gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);
-                gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);
-                commit_uni(&bar[B_RADONE]);
-                // Qt^T - Q^T = (-W)^T P^T over P0^T (which the out warps have turned into P^T),  OI^T = Uh^T P^T
-                if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
-                tc_fence_after();
-                gemm_uni<true, true, 64, N, N, N>(RC, x_b, pt_b);
-                gemm_uni<true, true, 64, N, N, N>(RD, v_b, pt_b);
-                commit_uni(&bar[B_D4DONE]);
+                ++ip3;
+                progress = true;
+            }
+            if (progress) {
+                t_last = clock64();
+            } else if (clock64() - t_last > WAIT_CYCLES) {
+                atomicCAS(err, 0, 142);
+                return;
+            } else if (*(volatile int*)err != 0) {
+                return;
             }
         }
-    } else {
+    } else if (warp == 12) {
+        // ------------------------------------------------ MMA issue, second warp: [E | Xi^T] -------------------------
+#pragma unroll 1
+        for (int k = 0; k < nk; ++k) {
+            const uint32_t x_b = smem_u32(smem + (k & 1) * F_REGION + X_OFF), v_b = x_b + V_OFF, k_b = x_b + K_OFF;
+            if (!PF_WAIT(B_WUREADY, k & 1, 149)) return;
+            tc_fence_after();
+            gemm_uni<true, true, DK, N, N, N>(RA, k_b, x_b);                        // E = K^T (-W)     (lanes i, columns i')
+            gemm_uni<true, true, DK, N, N, N>(RA + DK, v_b, k_b);                   // Xi^T = Uh^T K    (lanes j, columns i)
+            commit_uni(&bar[B_RADONE]);
+        }
+    } else if (warp == 15) {
+        // ------------------------------------------------ MMA issue, third warp: P0^T and [Qt^T | OI^T] --------------
+        const uint32_t q_b = smem_u32(smem + F_Q), pt_b = smem_u32(smem + F_PT), i16_b = smem_u32(smem + F_I16);
+#pragma unroll 1
+        for (int k = 0; k < nk; ++k) {
+            const uint32_t x_b = smem_u32(smem + (k & 1) * F_REGION + X_OFF), v_b = x_b + V_OFF, k_b = x_b + K_OFF;
+            // P0^T = K Q^T  (RC: Qt^T of the chunk before has been drained)
+            if (!PF_WAIT(B_K16 + (k & 1), (k >> 1) & 1, 152) || !PF_WAIT(B_Q16, k & 1, 153)) return;
+            if (k >= 1 && !PF_WAIT(B_D4FREE, (k - 1) & 1, 147)) return;
+            tc_fence_after();
+            gemm_uni<false, false, 64, DK, N, 64>(RC, k_b, q_b);
+            commit_uni(&bar[B_P0DONE]);
+            // Qt^T = Q^T + (-W)^T P^T (over P0^T, which the bulk warps have turned into P^T): Q^T first, 16 columns t at a
+            // time, as Q^T times a 16 x 16 identity (A = the Q tile read MN-major, one K-step of 16 tokens per block of
+            // columns);  OI^T = Uh^T P^T.   (All of the bulk warps have passed W / Uh on before they pass P^T on.)
+            if (!PF_WAIT(B_PTREADY, k & 1, 150)) return;
+            tc_fence_after();
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb)
+                gemm_lay<L_SWMN, L_NSK, 16, 16, 64, 16>(RC + 16 * cb, q_b + 2048 * cb, i16_b);
+            gemm_uni<true, true, 64, N, N, N, false, true>(RC, x_b, pt_b);
+            gemm_uni<true, true, 64, N, N, N>(RD, v_b, pt_b);
+            commit_uni(&bar[B_D4DONE]);
+        }
+    } else if (warp == 14) {
         // ------------------------------------------------ flag warp: ring back-pressure, ready flags ---------
         if (lane == 0) {
 #pragma unroll 1
@@ -676,7 +607,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = g.NC;
     int* err = ws.status;
-    const uint32_t t_delta = tb, t_o = tb + 128, t_a = tb + 256;     // Delta | 2 x O^T | 2 x fp16 state
+    const uint32_t t_delta = tb, t_o = tb + 256, t_a = tb + 384;     // 2 x (Xi^T + Delta) | 2 x O^T | 2 x fp16 state
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
     const int* ready = ws.ready + seq * 64;
@@ -688,6 +619,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
         // thread (w, j): row j of S, columns i = 64w .. 64w+63
         const int w = warp >> 2, j = tid & 127;
         float S[64];
+        int xi_issued = 0;      // (warp 0) steps whose Xi^T has been issued into its accumulator
         const long long sbase = ((long long)seq * DK + 64 * w) * DV + j;
 #pragma unroll
         for (int ii = 0; ii < 64; ++ii) S[ii] = S0 ? S0[sbase + (long long)ii * DV] : 0.f;
@@ -707,40 +639,52 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             }
             tc_fence_before();
             if (!named_bar_and(1, 256, ok)) return;
-            // warp 0 issues Delta[j][i] = sum_i' S[j][i'] E[i][i']; its completion also releases warp 13, which
-            // issues the O^T product of the same copy (so that O^T never sits in front of Delta in the tensor pipe)
+            // warp 0 issues Xi^T + Delta into accumulator c & 1, Delta[j][i] = sum_i' S[j][i'] E[i][i'].  Xi^T goes in first,
+            // as the fp16 image times a 16 x 16 identity, 16 columns per instruction (no state needed, so it is issued a
+            // step ahead whenever the image is there); Delta accumulates onto it.  The completion of Delta also releases
+            // warp 13, which issues the O^T product of the same copy (so that O^T never sits in front of Delta in the
+            // tensor pipe).
             if (warp == 0) {
+                const uint32_t i16_b = smem_u32(smem + F_I16);
+                if (xi_issued <= c) {
+                    if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
+                    tc_fence_after();
+                    const uint32_t xi_b = smem_u32(smem + S_XI + buf * 32768);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        gemm_lay<L_NSK, L_NSK, 16, 16, 128, 16>(t_delta + buf * 128 + 16 * kk, xi_b + 4096 * kk, i16_b);
+                    commit_uni(&bar[B_XIEMPTY + buf]);
+                    ++xi_issued;
+                }
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                gemm_ta<L_NSK, DK, DK, 128>(t_delta, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
+                gemm_ta<L_NSK, DK, DK, 128, true>(t_delta + buf * 128, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
                 commit_uni(&bar[B_APUB + buf]);
+                // Xi^T of the next step into the other accumulator (drained before this step's barrier), if its image is in
+                if (c + 1 < NC && mbar_test(&bar[B_XIFULL + (buf ^ 1)], ((c + 1) >> 1) & 1)) {
+                    tc_fence_after();
+                    const uint32_t xi_b = smem_u32(smem + S_XI + (buf ^ 1) * 32768);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        gemm_lay<L_NSK, L_NSK, 16, 16, 128, 16>(t_delta + (buf ^ 1) * 128 + 16 * kk, xi_b + 4096 * kk, i16_b);
+                    commit_uni(&bar[B_XIEMPTY + (buf ^ 1)]);
+                    ++xi_issued;
+                }
             }
-            if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
             if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
-            // S += Delta + Xi^T   (row j, columns 64w..64w+63; Xi^T from its column-group image)
-            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + j * 16;
+            // S += Xi^T + Delta   (row j, columns 64w..64w+63)
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
-                tmem_ld32(t_delta + lane_base + 64 * w + c0, rr);
-                uint4 xi[4];
-#pragma unroll
-                for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((c0 >> 3) + p) * 2048);
+                tmem_ld32(t_delta + buf * 128 + lane_base + 64 * w + c0, rr);
                 tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const uint32_t wd = ((const uint32_t*)&xi[e >> 3])[(e & 7) >> 1];
-                    const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&wd));
-                    S[c0 + e] += __uint_as_float(rr[e]) + xv.x;
-                    S[c0 + e + 1] += __uint_as_float(rr[e + 1]) + xv.y;
-                }
+                for (int e = 0; e < 32; ++e) S[c0 + e] += __uint_as_float(rr[e]);
             }
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
         }
         if (S_final)
 #pragma unroll
@@ -826,7 +770,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             commit_uni(&bar[B_QTEMPTY + buf]);
             commit_uni(&bar[B_S16FREE + buf]);
         }
-    } else {
+    } else if (warp == 14) {
         // ------------------------------------------------ ready flags in, consumed reports out -----------------
         // One lane polls the ring's ready flags in chunk order, as far ahead of the loads as the flow CTAs are, and
         // publishes the count in shared memory (so that no load waits a trip to the L2 for a flag that was set long
@@ -886,27 +830,27 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
         if (is_scan) {
             for (int x = 0; x < 2; ++x) {
                 mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
-                mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
+                mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 1);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
                 mbar_init(&bar[B_APUB + x], 1); mbar_init(&bar[B_S16FREE + x], 1);
                 mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
             }
         } else {
             for (int x = 0; x < 2; ++x) {
-                mbar_init(&bar[B_KFULL + x], 1); mbar_init(&bar[B_VFULL + x], 1);
-                mbar_init(&bar[B_K16 + x], 128); mbar_init(&bar[B_V16 + x], 128);
+                                mbar_init(&bar[B_KFULL + x], 1); mbar_init(&bar[B_VFULL + x], 1);
+                mbar_init(&bar[B_K16 + x], 256); mbar_init(&bar[B_V16 + x], 256);
                 mbar_init(&bar[B_XREADY + x], 128);
             }
-            mbar_init(&bar[B_QFULL], 1); mbar_init(&bar[B_Q16], 128);
-            mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128);
-            mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 256);
-            mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 128);
-            mbar_init(&bar[B_D4DONE], 1); mbar_init(&bar[B_RADONE], 1); mbar_init(&bar[B_D4FREE], 128); mbar_init(&bar[B_RAFREE], 256);
-            mbar_init(&bar[B_QCOPIED], 128); mbar_init(&bar[B_OUTDONE], 256);
-            mbar_init(&bar[B_SLOTOK], 1);
+            mbar_init(&bar[B_QFULL], 1); mbar_init(&bar[B_Q16], 256);
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.v);
+            mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128);
+            mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 256);
+            mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 256);
+            mbar_init(&bar[B_D4DONE], 1); mbar_init(&bar[B_RADONE], 1); mbar_init(&bar[B_D4FREE], 256); mbar_init(&bar[B_RAFREE], 256);
+            mbar_init(&bar[B_OUTDONE], 256);
+            mbar_init(&bar[B_SLOTOK], 1);
         }
         *(volatile int*)(smem + F_BAR + B_COUNT * 8 + 8) = 0;
         *(volatile int*)(smem + F_BAR + B_COUNT * 8 + 12) = 0;
@@ -916,8 +860,11 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
     if (!is_scan) {
         // operands with fewer than 128 rows are read past their tile: keep those bytes finite
         for (int e = tid; e < F_BETA / 16; e += FT) ((uint4*)smem)[e] = make_uint4(0, 0, 0, 0);
-        fence_async_smem();
     }
+    // a 16 x 16 fp16 identity, element (n, k) at ns_off(n, k, 16): the second operand of the products that add an fp16
+    // image to an accumulator (Q^T into Qt^T in the flow role, Xi^T into the state's increment in the scan role)
+    if (tid < 256) *(__half*)(smem + F_I16 + ns_off(tid >> 4, tid & 15, 16)) = __float2half_rn((tid >> 4) == (tid & 15) ? 1.f : 0.f);
+    fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();

@@ -62,75 +62,6 @@ struct FlowMaps {
     CUtensorMap q, k, v;
 };
 
-// One level of the recursive-doubling inverse: blocks of size S are merged into blocks of size 2S.
-// Task = (merge, 16-row strip); N/32 tasks per level, one warp each.
-template <int N, int S>
-__device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, int lane) {
-    constexpr int TASKS = N / 32;
-    constexpr int STRIPS = S / 16;
-    constexpr int NT = S / 8;       // n-tiles of 8 columns
-    float z[NT][4];
-    const bool has_task = warp < TASKS;
-    const int q = warp / STRIPS, strip = warp % STRIPS;
-    const int lo0 = 2 * S * q, hi0 = lo0 + S, R0 = hi0 + 16 * strip;
-    if (has_task) {
-        // U1[16 x S] = X[R0.., hi cols] * A[hi rows, lo cols]
-        float u[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) u[nt][e] = 0.f;
-#pragma unroll
-        for (int kk = 0; kk < S / 16; ++kk) {
-            if (kk > strip) continue;   // X_hi,hi is lower triangular: columns beyond this strip are zero
-            uint32_t a[4];
-            ldmatrix_x4(a, xb + slab_off(R0 + (lane & 15), hi0 + 16 * kk + ((lane >> 4) << 3), N));
-#pragma unroll
-            for (int np = 0; np < S / 16; ++np) {
-                uint32_t b[4];
-                const int id = lane >> 3;
-                ldmatrix_x4_trans(b, xb + slab_off(hi0 + 16 * kk + (lane & 7) + ((id & 1) << 3),
-                                                   lo0 + 16 * np + ((id >> 1) << 3), N));
-                mma_16816(u[2 * np], a, b[0], b[1]);
-                mma_16816(u[2 * np + 1], a, b[2], b[3]);
-            }
-        }
-        // Z[16 x S] = U1 * X[lo rows, lo cols]
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) z[nt][e] = 0.f;
-#pragma unroll
-        for (int kk = 0; kk < S / 16; ++kk) {
-            uint32_t a[4];
-            a[0] = pack_h2(u[2 * kk][0], u[2 * kk][1]);
-            a[1] = pack_h2(u[2 * kk][2], u[2 * kk][3]);
-            a[2] = pack_h2(u[2 * kk + 1][0], u[2 * kk + 1][1]);
-            a[3] = pack_h2(u[2 * kk + 1][2], u[2 * kk + 1][3]);
-#pragma unroll
-            for (int np = 0; np < S / 16; ++np) {
-                if (np > kk) continue;  // X_lo,lo is lower triangular: rows kk only reach columns <= kk
-                uint32_t b[4];
-                const int id = lane >> 3;
-                ldmatrix_x4_trans(b, xb + slab_off(lo0 + 16 * kk + (lane & 7) + ((id & 1) << 3),
-                                                   lo0 + 16 * np + ((id >> 1) << 3), N));
-                mma_16816(z[2 * np], a, b[0], b[1]);
-                mma_16816(z[2 * np + 1], a, b[2], b[3]);
-            }
-        }
-    }
-    __syncthreads();   // every strip has read A_hi,lo before anyone overwrites it
-    if (has_task) {
-        const int g = lane >> 2, t4 = lane & 3;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int col = lo0 + 8 * nt + 2 * t4;
-            *(uint32_t*)(xg + slab_off(R0 + g, col, N)) = pack_h2(-z[nt][0], -z[nt][1]);
-            *(uint32_t*)(xg + slab_off(R0 + g + 8, col, N)) = pack_h2(-z[nt][2], -z[nt][3]);
-        }
-    }
-    __syncthreads();
-}
 
 template <int N, int DK, int DV>
 __global__ void __launch_bounds__(FLOW_THREADS, (FlowSmem<N, DK, DV>::two_per_sm ? 2 : 1))
@@ -325,9 +256,9 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         __syncthreads();
         lap(4);
-        merge_level<N, 16>(x_b, sX, warp, lane);
-        merge_level<N, 32>(x_b, sX, warp, lane);
-        if (N == 128) merge_level<N, 64>(x_b, sX, warp, lane);
+        merge_level<N, 16, 0>(x_b, sX, warp, lane);
+        merge_level<N, 32, 0>(x_b, sX, warp, lane);
+        if (N == 128) merge_level<N, 64, 0>(x_b, sX, warp, lane);
 
         lap(5);
         // ---- T' = X diag(beta): the row owner scales its row by the column betas -----------------------------

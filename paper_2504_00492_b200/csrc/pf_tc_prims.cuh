@@ -50,6 +50,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Non-blocking test of a phase (try_wait may suspend the thread for a while; a poller of several barriers must not).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false (and raises *err_flag) if the phase never completes.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err_flag, int code) {
     for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
@@ -117,6 +127,13 @@ __device__ __forceinline__ uint4 ld_cg_u4(const void* p) {
     asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
+// Streaming 16-byte load of read-only input data (no L1 allocation).
+__device__ __forceinline__ uint4 ld_nc_u4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ float ld_cg_f32(const float* p) {
     float v;
     asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
@@ -212,6 +229,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }
@@ -346,7 +373,8 @@ __device__ __forceinline__ constexpr uint32_t kstep_off(int kk) {
          : LAY == L_SWMN ? (uint32_t)kk * 2048u
          : LAY == L_NSK ? (uint32_t)kk * 2u * (uint32_t)ROWS * 16u : (uint32_t)kk * 256u;
 }
-template <int AL, int BL, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
+// ACC: accumulate onto what the accumulator holds (from the first K-step on) instead of overwriting it.
+template <int AL, int BL, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false, bool ACC = false>
 __device__ __forceinline__ void gemm_lay(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
     constexpr bool A_MN = (AL == L_SWMN || AL == L_NSMN), B_MN = (BL == L_SWMN || BL == L_NSMN);
     constexpr uint32_t idesc = make_idesc(NCOLS, A_MN, B_MN, false) | (BF16 ? ((1u << 7) | (1u << 10)) : 0u);
@@ -354,11 +382,11 @@ __device__ __forceinline__ void gemm_lay(uint32_t d_tmem, uint32_t a_base, uint3
 #pragma unroll
     for (int kk = 0; kk < KDIM / 16; ++kk) {
         const uint64_t ad = a0 + (uint64_t)(kstep_off<AL, A_ROWS>(kk) >> 4), bd = b0 + (uint64_t)(kstep_off<BL, B_ROWS>(kk) >> 4);
-        if (elect_one()) mma_f16(d_tmem, ad, bd, idesc, kk > 0);
+        if (elect_one()) mma_f16(d_tmem, ad, bd, idesc, ACC || kk > 0);
     }
 }
 // D[128 x NCOLS] = A * B^T with A (fp16, K-major, KDIM/2 packed columns) in tensor memory; whole warp, converged.
-template <int BL, int NCOLS, int KDIM, int B_ROWS>
+template <int BL, int NCOLS, int KDIM, int B_ROWS, bool ACC = false>
 __device__ __forceinline__ void gemm_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base) {
     constexpr bool B_MN = (BL == L_SWMN || BL == L_NSMN);
     constexpr uint32_t idesc = make_idesc(NCOLS, false, B_MN, false);
@@ -366,12 +394,12 @@ __device__ __forceinline__ void gemm_ta(uint32_t d_tmem, uint32_t a_tmem, uint32
 #pragma unroll
     for (int kk = 0; kk < KDIM / 16; ++kk) {
         const uint64_t bd = b0 + (uint64_t)(kstep_off<BL, B_ROWS>(kk) >> 4);
-        if (elect_one()) mma_f16_ta(d_tmem, a_tmem + 8u * (uint32_t)kk, bd, idesc, kk > 0);
+        if (elect_one()) mma_f16_ta(d_tmem, a_tmem + 8u * (uint32_t)kk, bd, idesc, ACC || kk > 0);
     }
 }
-template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false>
+template <bool A_MN, bool B_MN, int NCOLS, int KDIM, int A_ROWS, int B_ROWS, bool BF16 = false, bool ACC = false>
 __device__ __forceinline__ void gemm_uni(uint32_t d_tmem, uint32_t a_base, uint32_t b_base) {
-    gemm_lay<A_MN ? L_SWMN : L_SWK, B_MN ? L_SWMN : L_SWK, NCOLS, KDIM, A_ROWS, B_ROWS, BF16>(d_tmem, a_base, b_base);
+    gemm_lay<A_MN ? L_SWMN : L_SWK, B_MN ? L_SWMN : L_SWK, NCOLS, KDIM, A_ROWS, B_ROWS, BF16, ACC>(d_tmem, a_base, b_base);
 }
 __device__ __forceinline__ void commit_uni(uint64_t* bar) {
     if (elect_one()) mma_commit(bar);
@@ -394,6 +422,154 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t sad
 __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
     __half2 h = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// byte offset of the 16-byte piece `col8` (= column / 8) of row `row` in a slab-stored matrix with R rows
+__device__ __forceinline__ uint32_t chunk_off(int row, int col8, int R) {
+    return (uint32_t)(col8 >> 3) * (uint32_t)R * 128u + (uint32_t)row * 128u + ((((uint32_t)col8 & 7u) ^ ((uint32_t)row & 7u)) << 4);
+}
+
+// ---- the triangular inverse X = (I + A)^{-1}, A strictly (block) lower triangular, fp16, slab-stored, N x N ----------
+// (Proposition on block-triangular inversion: diagonal blocks first, then off-diagonal blocks from them.)
+//
+// A 16 x 16 diagonal block by its Neumann product: A is nilpotent (A^16 = 0), so
+//     (I + A)^{-1} = (I - A)(I + A^2)(I + A^4)(I + A^8).
+// One warp, all in registers: the accumulator fragment of mma.m16n8k16 is, after packing to fp16, the A-operand
+// fragment of the same matrix, and the A-operand fragment of M^T serves as the two B-operand fragments of M, so the
+// powers are carried as the pair (M, M^T).  `deep`: include the A^8 factor (not needed when the mask groups rows in
+// pairs or more, since then A^8 = 0).  The block is read from and written back to rows/columns [16 blk, 16 blk + 16).
+__device__ __forceinline__ void frag_mul(float (&c)[2][4], const uint32_t (&x)[4], const uint32_t (&mt)[4]) {
+    mma_16816(c[0], x, mt[0], mt[2]);     // columns 0..7 of  X * M   (mt = A-operand fragment of M^T)
+    mma_16816(c[1], x, mt[1], mt[3]);     // columns 8..15
+}
+__device__ __forceinline__ void frag_pack(uint32_t (&f)[4], const float (&c)[2][4]) {
+    f[0] = pack_h2(c[0][0], c[0][1]);
+    f[1] = pack_h2(c[0][2], c[0][3]);
+    f[2] = pack_h2(c[1][0], c[1][1]);
+    f[3] = pack_h2(c[1][2], c[1][3]);
+}
+__device__ __forceinline__ void frag_zero(float (&c)[2][4]) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c[h][e] = 0.f;
+}
+__device__ __forceinline__ void diag_inverse16(uint32_t xb, uint8_t* xg, int blk, int lane, int N, bool deep) {
+    const int R0 = 16 * blk, c8 = 2 * blk;
+    uint32_t a[4], at[4];
+    ldmatrix_x4(a, xb + chunk_off(R0 + (lane & 15), c8 + (lane >> 4), N));
+    ldmatrix_x4_trans(at, xb + chunk_off(R0 + (lane & 7) + ((lane >> 4) << 3), c8 + ((lane >> 3) & 1), N));
+    float c[2][4], ct[2][4];
+    uint32_t a2[4], a2t[4], a4[4], a4t[4];
+    frag_zero(c); frag_zero(ct);
+    frag_mul(c, a, at);         // A^2
+    frag_mul(ct, at, a);        // (A^2)^T = A^T A^T
+    frag_pack(a2, c); frag_pack(a2t, ct);
+    frag_zero(c); frag_zero(ct);
+    frag_mul(c, a2, a2t);       // A^4
+    frag_mul(ct, a2t, a2);
+    frag_pack(a4, c); frag_pack(a4t, ct);
+    // R = I - A in accumulator layout: thread (g, t) holds rows g, g+8 and columns 8h + 2t, 8h + 2t + 1
+    const int gq = lane >> 2, t4 = lane & 3;
+    float r[2][4];
+    {
+        const __half2 h0 = *reinterpret_cast<const __half2*>(&a[0]), h1 = *reinterpret_cast<const __half2*>(&a[1]);
+        const __half2 h2 = *reinterpret_cast<const __half2*>(&a[2]), h3 = *reinterpret_cast<const __half2*>(&a[3]);
+        const float2 f0 = __half22float2(h0), f1 = __half22float2(h1), f2 = __half22float2(h2), f3 = __half22float2(h3);
+        const float d0 = (gq == 2 * t4) ? 1.f : 0.f, d1 = (gq == 2 * t4 + 1) ? 1.f : 0.f;
+        r[0][0] = d0 - f0.x; r[0][1] = d1 - f0.y;     // row g,   columns 2t, 2t+1
+        r[0][2] = -f1.x;     r[0][3] = -f1.y;         // row g+8, columns 2t, 2t+1
+        r[1][0] = -f2.x;     r[1][1] = -f2.y;         // row g,   columns 8+2t, 8+2t+1
+        r[1][2] = d0 - f3.x; r[1][3] = d1 - f3.y;     // row g+8, columns 8+2t, 8+2t+1
+    }
+    uint32_t rf[4];
+    frag_pack(rf, r);
+    frag_mul(r, rf, a2t);       // R (I + A^2)
+    frag_pack(rf, r);
+    frag_mul(r, rf, a4t);       // ... (I + A^4)
+    if (deep) {
+        frag_zero(ct);
+        frag_mul(ct, a4t, a4);  // (A^8)^T
+        uint32_t a8t[4];
+        frag_pack(a8t, ct);
+        frag_pack(rf, r);
+        frag_mul(r, rf, a8t);   // ... (I + A^8)
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        *(uint32_t*)(xg + chunk_off(R0 + gq, c8 + h, N) + 4 * t4) = pack_h2(r[h][0], r[h][1]);
+        *(uint32_t*)(xg + chunk_off(R0 + gq + 8, c8 + h, N) + 4 * t4) = pack_h2(r[h][2], r[h][3]);
+    }
+}
+
+// One level of the recursive-doubling inverse: diagonal blocks of size S are merged into blocks of size 2S,
+//     X_hi,lo = -X_hi,hi A_hi,lo X_lo,lo.
+// Task = (merge, 16-row strip): N/32 tasks, one warp each; the four warps synchronise on named barrier BAR
+// (128 threads; BAR = 0 is the CTA barrier of a 128-thread CTA).
+template <int N, int S, int BAR>
+__device__ __forceinline__ void merge_level(uint32_t xb, uint8_t* xg, int warp, int lane) {
+    constexpr int TASKS = N / 32;
+    constexpr int STRIPS = S / 16;
+    constexpr int NT = S / 8;
+    float z[NT][4];
+    const bool has_task = warp < TASKS;
+    const int q = warp / STRIPS, strip = warp % STRIPS;
+    const int lo0 = 2 * S * q, hi0 = lo0 + S, R0 = hi0 + 16 * strip;
+    const int id = lane >> 3;
+    if (has_task) {
+        float u[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) u[nt][e] = 0.f;
+        // (all column offsets below are multiples of 8, all row offsets multiples of 8 plus a lane term)
+        const int a_row = R0 + (lane & 15), a_c8 = (hi0 >> 3) + (lane >> 4);
+        const int b_rowl = (lane & 7) + ((id & 1) << 3), b_c8l = (id >> 1);
+#pragma unroll
+        for (int kk = 0; kk < S / 16; ++kk) {
+            if (kk > strip) continue;   // X_hi,hi is lower triangular
+            uint32_t a[4];
+            ldmatrix_x4(a, xb + chunk_off(a_row, a_c8 + 2 * kk, N));
+#pragma unroll
+            for (int np = 0; np < S / 16; ++np) {
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, xb + chunk_off(hi0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
+                mma_16816(u[2 * np], a, b[0], b[1]);
+                mma_16816(u[2 * np + 1], a, b[2], b[3]);
+            }
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) z[nt][e] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < S / 16; ++kk) {
+            uint32_t a[4];
+            a[0] = pack_h2(u[2 * kk][0], u[2 * kk][1]);
+            a[1] = pack_h2(u[2 * kk][2], u[2 * kk][3]);
+            a[2] = pack_h2(u[2 * kk + 1][0], u[2 * kk + 1][1]);
+            a[3] = pack_h2(u[2 * kk + 1][2], u[2 * kk + 1][3]);
+#pragma unroll
+            for (int np = 0; np < S / 16; ++np) {
+                if (np > kk) continue;  // X_lo,lo is lower triangular
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, xb + chunk_off(lo0 + 16 * kk + b_rowl, (lo0 >> 3) + 2 * np + b_c8l, N));
+                mma_16816(z[2 * np], a, b[0], b[1]);
+                mma_16816(z[2 * np + 1], a, b[2], b[3]);
+            }
+        }
+    }
+    named_bar(BAR, 128);   // every strip has read A_hi,lo before anyone overwrites it
+    if (has_task) {
+        const int gq = lane >> 2, t4 = lane & 3;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int c8 = (lo0 >> 3) + nt;
+            *(uint32_t*)(xg + chunk_off(R0 + gq, c8, N) + 4 * t4) = pack_h2(-z[nt][0], -z[nt][1]);
+            *(uint32_t*)(xg + chunk_off(R0 + gq + 8, c8, N) + 4 * t4) = pack_h2(-z[nt][2], -z[nt][3]);
+        }
+    }
+    named_bar(BAR, 128);
 }
 
 }  // namespace tc
