@@ -370,16 +370,19 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 const float bm = h ? -bs : bs;
                 uint8_t* mrow = smem + b * F_REGION + (h ? X_OFF : V_OFF) + m * 128;
                 const uint32_t src = RA + lane_base + h * 128;
+                // (a tensor-memory load and its wait cost the same ~170 cycles whatever the width: two 32-column loads per wait)
 #pragma unroll 1
                 for (int sl = 0; sl < 2; ++sl) {                 // 64-column slab
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(src + 64 * sl, ra);
+                    tmem_ld32(src + 64 * sl + 32, rb);
+                    tmem_ld_wait();
+                    if (m < N) {
+                        uint8_t* base = mrow + sl * (N * 128);
 #pragma unroll
-                    for (int st4 = 0; st4 < 4; ++st4) {          // 16 columns = two 16-byte pieces
-                        uint32_t rr[16];
-                        tmem_ld16(src + 64 * sl + 16 * st4, rr);
-                        tmem_ld_wait();
-                        if (m < N) {
-                            *(uint4*)(mrow + sl * (N * 128) + (((uint32_t)(2 * st4) << 4) ^ sw16)) = pack8(rr, bm);
-                            *(uint4*)(mrow + sl * (N * 128) + (((uint32_t)(2 * st4 + 1) << 4) ^ sw16)) = pack8(rr + 8, bm);
+                        for (int j8 = 0; j8 < 4; ++j8) {
+                            *(uint4*)(base + (((uint32_t)j8 << 4) ^ sw16)) = pack8(ra + 8 * j8, bm);
+                            *(uint4*)(base + (((uint32_t)(j8 + 4) << 4) ^ sw16)) = pack8(rb + 8 * j8, bm);
                         }
                     }
                 }
@@ -394,24 +397,21 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             {
                 const int lo = m < nv ? tokm : 64;               // tokens t in [lo, Cv) see row m
                 uint8_t* prow_ = smem + F_PT + m * 128;          // (one slab: 64 columns)
+                const int c0 = 32 * h;
+                uint32_t rr[32];
+                tmem_ld32(RC + lane_base + c0, rr);
+                tmem_ld_wait();
+                if (m < N) {
 #pragma unroll
-                for (int st2 = 0; st2 < 2; ++st2) {
-                    const int c0 = 32 * h + 16 * st2;
-                    uint32_t rr[16];
-                    tmem_ld16(RC + lane_base + c0, rr);
-                    tmem_ld_wait();
-                    if (m < N) {
+                    for (int j8 = 0; j8 < 32; j8 += 8) {
+                        float a[8];
 #pragma unroll
-                        for (int j8 = 0; j8 < 16; j8 += 8) {
-                            float a[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int t = c0 + j8 + j;
-                                a[j] = (t >= lo && t < Cv) ? __uint_as_float(rr[j8 + j]) : 0.f;
-                            }
-                            *(uint4*)(prow_ + (((uint32_t)((c0 + j8) >> 3) << 4) ^ sw16)) =
-                                make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
+                        for (int j = 0; j < 8; ++j) {
+                            const int t = c0 + j8 + j;
+                            a[j] = (t >= lo && t < Cv) ? __uint_as_float(rr[j8 + j]) : 0.f;
                         }
+                        *(uint4*)(prow_ + (((uint32_t)((c0 + j8) >> 3) << 4) ^ sw16)) =
+                            make_uint4(pack_h2(a[0], a[1]), pack_h2(a[2], a[3]), pack_h2(a[4], a[5]), pack_h2(a[6], a[7]));
                     }
                 }
             }
@@ -428,13 +428,14 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                 const uint32_t src = RA + lane_base + (h ? 0 : DK);
 #pragma unroll 1
                 for (int sl = 0; sl < 2; ++sl) {
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(src + 64 * sl, ra);
+                    tmem_ld32(src + 64 * sl + 32, rb);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int st4 = 0; st4 < 4; ++st4) {
-                        uint32_t rr[16];
-                        tmem_ld16(src + 64 * sl + 16 * st4, rr);
-                        tmem_ld_wait();
-                        *(uint4*)(row + sl * 16384 + (2 * st4) * 2048) = pack8n(rr);
-                        *(uint4*)(row + sl * 16384 + (2 * st4 + 1) * 2048) = pack8n(rr + 8);
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        *(uint4*)(row + sl * 16384 + j8 * 2048) = pack8n(ra + 8 * j8);
+                        *(uint4*)(row + sl * 16384 + (j8 + 4) * 2048) = pack8n(rb + 8 * j8);
                     }
                 }
             }
@@ -459,37 +460,33 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                     load_v(b, s2, c2);
                 }
             }
-            if (h == 1) {
-                uint8_t* qrow = slot + SLOT_QT + m * 16;
+            {
+                uint32_t ra[32], rb[32];
+                const uint32_t src = (h ? RC : RD) + lane_base;
+                tmem_ld32(src, ra);
+                tmem_ld32(src + 32, rb);
+                tmem_ld_wait();
+                if (h == 1) {
+                    uint8_t* qrow = slot + SLOT_QT + m * 16;
 #pragma unroll
-                for (int st4 = 0; st4 < 4; ++st4) {
-                    uint32_t rr[16];
-                    tmem_ld16(RC + lane_base + 16 * st4, rr);
-                    tmem_ld_wait();
-                    *(uint4*)(qrow + (2 * st4) * 2048) = pack8n(rr);
-                    *(uint4*)(qrow + (2 * st4 + 1) * 2048) = pack8n(rr + 8);
-                }
-            } else {
-                float* oi = O + ((long long)seq * g.L + (long long)c * C) * DV + m;
-                if (Cv == 64) {
-#pragma unroll
-                    for (int st4 = 0; st4 < 4; ++st4) {
-                        uint32_t rr[16];
-                        tmem_ld16(RD + lane_base + 16 * st4, rr);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) oi[(16 * st4 + j) * DV] = __uint_as_float(rr[j]);
+                    for (int j8 = 0; j8 < 4; ++j8) {
+                        *(uint4*)(qrow + j8 * 2048) = pack8n(ra + 8 * j8);
+                        *(uint4*)(qrow + (j8 + 4) * 2048) = pack8n(rb + 8 * j8);
                     }
                 } else {
-#pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
-                        uint32_t rr[16];
-                        tmem_ld16(RD + lane_base + c0, rr);
-                        tmem_ld_wait();
-                        const int lim = Cv - c0;
+                    float* oi = O + ((long long)seq * g.L + (long long)c * C) * DV + m;
+                    if (Cv == 64) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (j < lim) oi[(c0 + j) * DV] = __uint_as_float(rr[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            oi[j * DV] = __uint_as_float(ra[j]);
+                            oi[(32 + j) * DV] = __uint_as_float(rb[j]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < Cv) oi[j * DV] = __uint_as_float(ra[j]);
+                            if (32 + j < Cv) oi[(32 + j) * DV] = __uint_as_float(rb[j]);
+                        }
                     }
                 }
             }
