@@ -129,7 +129,7 @@ enum {
     B_EFULL = 32,     // [2] producer: E image landed
     B_EEMPTY = 34,    // [2] chain: Delta of that chunk complete
     B_XIFULL = 36,    // [2] producer: Xi image landed
-    B_XIEMPTY = 38,   // [2] mma: the Xi image has been read into its accumulator
+    B_XIEMPTY = 38,   // [2] chain: Xi added to the state (one arrival per chain warp)
     B_QTFULL = 40,    // [2] producer: Qt image landed
     B_QTEMPTY = 42,   // [2] mma: O^T of that chunk complete
     B_APUB = 44,      // [2 buffers] mma: Delta of the chunk complete (the O^T product may be issued)
@@ -604,7 +604,7 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = g.NC;
     int* err = ws.status;
-    const uint32_t t_delta = tb, t_o = tb + 256, t_a = tb + 384;     // 2 x (Xi^T + Delta) | 2 x O^T | 2 x fp16 state
+    const uint32_t t_delta = tb, t_o = tb + 128, t_a = tb + 256;     // Delta | 2 x O^T | 2 x fp16 state
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint8_t* ring = ws.ring + (size_t)seq * g.R * SLOT_BYTES;
     const int* ready = ws.ready + seq * 64;
@@ -616,7 +616,6 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
         // thread (w, j): row j of S, columns i = 64w .. 64w+63
         const int w = warp >> 2, j = tid & 127;
         float S[64];
-        int xi_issued = 0;      // (warp 0) steps whose Xi^T has been issued into its accumulator
         const long long sbase = ((long long)seq * DK + 64 * w) * DV + j;
 #pragma unroll
         for (int ii = 0; ii < 64; ++ii) S[ii] = S0 ? S0[sbase + (long long)ii * DV] : 0.f;
@@ -636,52 +635,40 @@ __device__ void scan_role(const FusedGeo& g, const FusedWs& ws, const float* __r
             }
             tc_fence_before();
             if (!named_bar_and(1, 256, ok)) return;
-            // warp 0 issues Xi^T + Delta into accumulator c & 1, Delta[j][i] = sum_i' S[j][i'] E[i][i'].  Xi^T goes in first,
-            // as the fp16 image times a 16 x 16 identity, 16 columns per instruction (no state needed, so it is issued a
-            // step ahead whenever the image is there); Delta accumulates onto it.  The completion of Delta also releases
-            // warp 13, which issues the O^T product of the same copy (so that O^T never sits in front of Delta in the
-            // tensor pipe).
+            // warp 0 issues Delta[j][i] = sum_i' S[j][i'] E[i][i']; its completion also releases warp 13, which
+            // issues the O^T product of the same copy (so that O^T never sits in front of Delta in the tensor pipe)
             if (warp == 0) {
-                const uint32_t i16_b = smem_u32(smem + F_I16);
-                if (xi_issued <= c) {
-                    if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
-                    tc_fence_after();
-                    const uint32_t xi_b = smem_u32(smem + S_XI + buf * 32768);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        gemm_lay<L_NSK, L_NSK, 16, 16, 128, 16>(t_delta + buf * 128 + 16 * kk, xi_b + 4096 * kk, i16_b);
-                    commit_uni(&bar[B_XIEMPTY + buf]);
-                    ++xi_issued;
-                }
                 if (!PF_WAIT(B_EFULL + buf, (c >> 1) & 1, 231)) return;
                 tc_fence_after();
-                gemm_ta<L_NSK, DK, DK, 128, true>(t_delta + buf * 128, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
+                gemm_ta<L_NSK, DK, DK, 128>(t_delta, t_a + buf * 64, smem_u32(smem + S_E + buf * 32768));
                 commit_uni(&bar[B_DDONE]);
                 commit_uni(&bar[B_EEMPTY + buf]);
                 commit_uni(&bar[B_APUB + buf]);
-                // Xi^T of the next step into the other accumulator (drained before this step's barrier), if its image is in
-                if (c + 1 < NC && mbar_test(&bar[B_XIFULL + (buf ^ 1)], ((c + 1) >> 1) & 1)) {
-                    tc_fence_after();
-                    const uint32_t xi_b = smem_u32(smem + S_XI + (buf ^ 1) * 32768);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        gemm_lay<L_NSK, L_NSK, 16, 16, 128, 16>(t_delta + (buf ^ 1) * 128 + 16 * kk, xi_b + 4096 * kk, i16_b);
-                    commit_uni(&bar[B_XIEMPTY + (buf ^ 1)]);
-                    ++xi_issued;
-                }
             }
+            if (!PF_WAIT(B_XIFULL + buf, (c >> 1) & 1, 203)) return;
             if (!PF_WAIT(B_DDONE, c & 1, 202)) return;
             tc_fence_after();
-            // S += Xi^T + Delta   (row j, columns 64w..64w+63)
+            // S += Delta + Xi^T   (row j, columns 64w..64w+63; Xi^T from its column-group image)
+            const uint8_t* xrow = smem + S_XI + buf * 32768 + w * 16384 + j * 16;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t rr[32];
-                tmem_ld32(t_delta + buf * 128 + lane_base + 64 * w + c0, rr);
+                tmem_ld32(t_delta + lane_base + 64 * w + c0, rr);
+                uint4 xi[4];
+#pragma unroll
+                for (int p = 0; p < 4; ++p) xi[p] = *(const uint4*)(xrow + ((c0 >> 3) + p) * 2048);
                 tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) S[c0 + e] += __uint_as_float(rr[e]);
+                for (int e = 0; e < 32; e += 2) {
+                    const uint32_t wd = ((const uint32_t*)&xi[e >> 3])[(e & 7) >> 1];
+                    const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&wd));
+                    S[c0 + e] += __uint_as_float(rr[e]) + xv.x;
+                    S[c0 + e + 1] += __uint_as_float(rr[e + 1]) + xv.y;
+                }
             }
             tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar[B_XIEMPTY + buf]);
         }
         if (S_final)
 #pragma unroll
@@ -827,7 +814,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
         if (is_scan) {
             for (int x = 0; x < 2; ++x) {
                 mbar_init(&bar[B_EFULL + x], 1); mbar_init(&bar[B_EEMPTY + x], 1);
-                mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 1);
+                mbar_init(&bar[B_XIFULL + x], 1); mbar_init(&bar[B_XIEMPTY + x], 8);
                 mbar_init(&bar[B_QTFULL + x], 1); mbar_init(&bar[B_QTEMPTY + x], 1);
                 mbar_init(&bar[B_APUB + x], 1); mbar_init(&bar[B_S16FREE + x], 1);
                 mbar_init(&bar[B_DDONE + x], 1); mbar_init(&bar[B_ODONE + x], 1); mbar_init(&bar[B_OFREE + x], 128);
