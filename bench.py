@@ -255,6 +255,61 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+class SlicePipeline:
+    """End-to-end step over slices of the (b,h) sequences on three streams (copy in, compute, copy out).
+
+    All tensors are [B, H, ...] contiguous, so a run of consecutive (b,h) sequences is one contiguous range; a slice is
+    handed to the library as a batch of its own (B = 1, H = sequences in the slice).  Per slice: the copy in waits for
+    the previous step's kernel on that slice (its device buffers are reused), the kernel waits for the copy in and for
+    the previous copy out of that slice's O, the copy out waits for the kernel."""
+
+    def __init__(self, host, dev, O, Sf, hO, hS, w, forward, n_slices):
+        self.w, self.forward = w, forward
+        n_seq = w.B * w.H
+        per = (n_seq + n_slices - 1) // n_slices
+        self.ranges = [(a, min(a + per, n_seq)) for a in range(0, n_seq, per)]
+        self.n = len(self.ranges)
+        flat = lambda t: None if t is None else t.reshape((n_seq,) + tuple(t.shape[2:]))
+        self.h = [flat(t) for t in (host.q, host.k, host.v, host.beta, host.S0)]
+        self.d = [flat(t) for t in (dev.q, dev.k, dev.v, dev.beta, dev.S0)]
+        self.O, self.Sf, self.hO, self.hS = flat(O), flat(Sf), flat(hO), flat(hS)
+        self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        self.in_done = [torch.cuda.Event() for _ in self.ranges]
+        self.k_done = [torch.cuda.Event() for _ in self.ranges]
+        self.out_done = [torch.cuda.Event() for _ in self.ranges]
+        self.first = True
+
+    def step(self, stream):
+        """One pass over all slices; `stream` (the timing stream) does the compute and joins the copy streams."""
+        start = torch.cuda.Event()
+        start.record(stream)
+        self.s_in.wait_event(start)
+        self.s_out.wait_event(start)
+        for i, (a, b) in enumerate(self.ranges):
+            with torch.cuda.stream(self.s_in):
+                if not self.first:
+                    self.s_in.wait_event(self.k_done[i])
+                for hs, ds in zip(self.h, self.d):
+                    if hs is not None:
+                        ds[a:b].copy_(hs[a:b], non_blocking=True)
+                self.in_done[i].record(self.s_in)
+            stream.wait_event(self.in_done[i])
+            if not self.first:
+                stream.wait_event(self.out_done[i])
+            sl = lambda t: None if t is None else t[a:b].unsqueeze(0)
+            q, k, v, beta, S0 = (sl(t) for t in self.d)
+            self.forward(q, k, v, beta, S0, O=sl(self.O), S_final=sl(self.Sf), stream=stream)
+            self.k_done[i].record(stream)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(self.k_done[i])
+                self.hO[a:b].copy_(self.O[a:b], non_blocking=True)
+                self.hS[a:b].copy_(self.Sf[a:b], non_blocking=True)
+                self.out_done[i].record(self.s_out)
+        stream.wait_event(self.in_done[-1])
+        stream.wait_event(self.out_done[-1])
+        self.first = False
+
+
 def kernel_profile(pf, d, w, steps):
     """Per-kernel device time (ms per launch, averaged) from CUDA events recorded inside the library."""
     from paper_2504_00492_b200 import binding
@@ -287,8 +342,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures)")
     ap.add_argument("--heads", type=int, default=0, help="override H of the workload (profiling captures)")
-    ap.add_argument("--ring-depth", type=int, default=0, help="pf_set_option('ring_depth', N) before running")
-    ap.add_argument("--segments", type=int, default=0, help="pf_set_option('segments', N) before running")
+    ap.add_argument("--ring-depth", type=int, default=0, help="pf_params.ring_depth (0 = the library's default)")
+    ap.add_argument("--segments", type=int, default=0, help="pf_params.segments (0 = the library's default)")
+    ap.add_argument("--e2e-slices", type=int, default=8, help="(b,h) slices of the pipelined end-to-end run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pf_synth.CONFIGS[args.workload]
@@ -307,11 +363,22 @@ def main():
     rank, world, local = ranks.rank, ranks.world, ranks.local
 
     import paper_2504_00492_b200 as pf
-    if args.ring_depth:
-        pf.pf_set_option("ring_depth", args.ring_depth)
-    if args.segments:
-        pf.pf_set_option("segments", args.segments)
     peaks, peak_kind = load_peaks()
+    options = {}
+    if args.ring_depth:
+        options["ring_depth"] = args.ring_depth
+    if args.segments:
+        options["segments"] = args.segments
+    in_dtype = pf.PF_DTYPE_F32 if w.dtype == "f32" else pf.PF_DTYPE_BF16
+    # PF_IMPL_AUTO may evaluate with a shorter chunk than the one asked for (the recurrence's result does not depend
+    # on it); the work counts below use the chunk length the kernels ran with.
+    chunk_used = pf.pf_select_chunk(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, in_dtype)
+    w_eval = w.with_(chunk=chunk_used)
+
+    def forward(q, k, v, beta, S0, O=None, S_final=None, stream=None):
+        if options:
+            return pf.pf_deltanet_fwd_ex(q, k, v, beta, S0, w.chunk, O=O, S_final=S_final, stream=stream, **options)
+        return fwd_of(pf, w)(q, k, v, beta, S0, w.chunk, O=O, S_final=S_final, stream=stream)
 
     host = pf_synth.make_inputs(w, seed=ranks.seed(w.seed)).pin()
     d = host.to("cuda")
@@ -320,7 +387,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        fwd_of(pf, w)(d.q, d.k, d.v, d.beta, d.S0, w.chunk, O=O, S_final=Sf)
+        forward(d.q, d.k, d.v, d.beta, d.S0, O=O, S_final=Sf)
 
     barrier = ranks.barrier
 
@@ -348,13 +415,17 @@ def main():
     value = tokens_per_step * args.steps / (total_ms * 1e-3)
 
     # ---- end to end: pinned host inputs -> device, call, outputs -> pinned host, all timed --------------
+    # (a) serial: one copy in, one call, one copy out per step, all on one stream;
+    # (b) pipelined: the (b,h) sequences are independent, so the batch is cut into slices and slice i's copy in,
+    #     call and copy out run on three streams, chained by events: the copies of one slice overlap the kernel of
+    #     another and the two copy directions overlap each other.  The reported e2e value is (b)'s.
     hO = torch.empty(O.shape, dtype=O.dtype).pin_memory()
     hS = torch.empty(Sf.shape, dtype=Sf.dtype).pin_memory()
     e2e_steps = max(3, min(args.steps, 10))
 
     def e2e_step():
         dd = host.to("cuda", non_blocking=True)
-        o, s = fwd_of(pf, w)(dd.q, dd.k, dd.v, dd.beta, dd.S0, w.chunk, O=O, S_final=Sf)
+        o, s = forward(dd.q, dd.k, dd.v, dd.beta, dd.S0, O=O, S_final=Sf)
         hO.copy_(o, non_blocking=True)
         hS.copy_(s, non_blocking=True)
 
@@ -366,18 +437,30 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = ranks.max_over_ranks(e2e_ms)
-    e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3)
+    e2e_serial_ms = ranks.max_over_ranks(e0.elapsed_time(e1))
+    e2e_serial = tokens_per_step * e2e_steps / (e2e_serial_ms * 1e-3)
     h2d = host.nbytes()
     d2h = hO.numel() * 4 + hS.numel() * 4
 
+    pipe = SlicePipeline(host, d, O, Sf, hO, hS, w, forward, max(1, min(args.e2e_slices, w.B * w.H)))
+    pipe.step(stream)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        pipe.step(stream)
+    e1.record(stream)
+    barrier()
+    e2e_ms = ranks.max_over_ranks(e0.elapsed_time(e1))
+    e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3)
+    e2e_launches = pf.pf_last_launch_count() * pipe.n
+
     # ---- per-kernel times and the roofline of the dominant kernel -----------------------------------------
     prof = kernel_profile(pf, d, w, steps=min(args.steps, 5))
-    G = w.B * w.H * ((w.L + w.chunk - 1) // w.chunk)
+    G = w.B * w.H * ((w.L + chunk_used - 1) // chunk_used)
     th = w.token_heads
-    fl_tri = flops_per_chunk(w, tri=True)
-    fl_dense = flops_per_chunk(w, tri=False)
+    fl_tri = flops_per_chunk(w_eval, tri=True)
+    fl_dense = flops_per_chunk(w_eval, tri=False)
     ms_step = total_ms / args.steps
     t_hbm_us = th * alg_bytes_per_token_head(w) / (peaks["hbm_gbs"] * 1e9) * 1e6
     t_flop_us = G * sum(fl_dense[k] for k in fl_dense if k != "solve") / (peaks["bf16_tflops"] * 1e12) * 1e6
@@ -431,12 +514,16 @@ def main():
                 w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk) == pf.PF_IMPL_TC else "f32",
             "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_k": w.d_k, "d_v": w.d_v, "r": w.r,
-                       "chunk": w.chunk, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
+                       "chunk": w.chunk, "chunk_evaluated": chunk_used, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
                            (host.nbytes() + O.numel() * 4) / 1e6), "parallelism": "replicas" if world > 1 else "1 GPU"},
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
             "token_heads_per_s": value * w.H,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps},
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                    "how": "%d (b,h) slices pipelined on 3 streams (copy in, compute, copy out)" % pipe.n,
+                    "launches_per_step": e2e_launches,
+                    "serial": {"value": e2e_serial, "ms_per_step": e2e_serial_ms / e2e_steps,
+                               "how": "one copy in, one call, one copy out per step on one stream"}},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
             "path_roofline": path, "cpu_baseline": cpu,
         }

@@ -25,7 +25,7 @@
  *   - Tensor pointers are DEVICE pointers owned by the caller, dense row-major in the shapes given;
  *     the library neither frees nor keeps them.  q/k/v/beta/O must be 16-byte aligned.
  *   - `stream` is a cudaStream_t (NULL = the default stream).  Work is enqueued; the calls do not
- *     synchronise.  Unless a workspace is passed through pf_deltanet_fwd_ex, scratch memory is
+ *     synchronise (pf_read_status and pf_profile_read do).  Unless a workspace is passed through pf_deltanet_fwd_ex, scratch memory is
  *     taken and returned with stream-ordered allocation on `stream`.
  *   - O must not alias an input.  S_final may alias S0.
  *   - Return value: PF_OK (0) or a negative pf_status.  Nothing is launched when an argument check
@@ -51,7 +51,7 @@ typedef enum pf_status {
     PF_ERR_ARCH = -4,         /* current device is not compute capability 10.x */
     PF_ERR_CUDA = -5,         /* a CUDA runtime call failed; see pf_last_error_string() */
     PF_ERR_WORKSPACE = -6,    /* caller workspace too small or misaligned */
-    PF_ERR_TIMEOUT = -7       /* a bounded device-side wait expired (reported via status word) */
+    PF_ERR_TIMEOUT = -7       /* a bounded device-side wait expired; returned by pf_read_status (see there) */
 } pf_status;
 
 enum { PF_DTYPE_BF16 = 0, PF_DTYPE_F32 = 1 };
@@ -86,8 +86,8 @@ enum { PF_STEP_EULER = 0, PF_STEP_EXACT = 1 };
  *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.  The result does
  *                  not depend on the chunk length beyond rounding, so AUTO may evaluate with another supported
  *                  chunk length than the one passed when that puts the problem on the tensor-core kernels (64 or
- *                  128 rows per chunk: e.g. r = 4 with chunk 64 runs as chunk 32).  The explicit choices below
- *                  use `chunk` as given.
+ *                  128 rows per chunk: e.g. r = 4 with chunk 64 runs as chunk 32; pf_select_chunk tells which).  The
+ *                  explicit choices below use `chunk` as given.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
  *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.  For
  *                  d_k = d_v = 128 with at most (SM count - 8) sequences this is ONE cooperative launch in
@@ -111,6 +111,12 @@ enum { PF_IMPL_AUTO = 0, PF_IMPL_SIMT = 1, PF_IMPL_TC = 2,
  *   S_final [B,H,d_k,d_v] fp32 or NULL (not wanted)   (written)
  * Defined by: recurrence/readout of Section 1.1, delta rule of Section 1.3, rank-R drivers of
  * Section 3.1, evaluated per chunk through Theorem 3.2 and carried across chunks (Section 3).
+ * Value range: the tensor-core kernels round q, k, v, the per-chunk operands derived from them and, once per chunk,
+ * the state S to fp16 before each product (fp32 accumulation).  fp16 has the 8 significant bits of bf16 and more, but
+ * only the exponent range 6.1e-5 .. 65504: an element of v, S0 or of the running state beyond 65504 in magnitude becomes
+ * infinite without an error code, and elements below 6.1e-5 lose precision gradually.  The stated tolerance (2e-3 of
+ * max|O|) is tested for |v|, |S| up to the order of 1e3.  The operation is linear in (v, S0): scale them by a power
+ * of two and O, S_final back for data outside that range, or ask for PF_IMPL_SIMT (fp32 throughout, no such limit).
  */
 int pf_deltanet_fwd(const void* q, const void* k, const void* v, const void* beta, const float* S0,
                     int B, int H, int L, int d_k, int d_v, int r, int chunk,
@@ -131,8 +137,9 @@ int pf_deltanet_fwd_f32(const float* q, const float* k, const float* v, const fl
  * per-chunk scratch from the stream-ordered allocator or from the caller; this one uses a fixed array
  * of PF_STATIC_SCRATCH_BYTES that is part of the library image, so it calls no allocating routine.
  *
- *   - Arguments, layouts, results and error codes are those of pf_deltanet_fwd_f32.
- *   - A problem whose scratch (pf_workspace_bytes(..., PF_DTYPE_F32, PF_IMPL_SIMT)) exceeds
+ *   - Arguments, layouts, results, checks and error codes are those of pf_deltanet_fwd_f32 (the fp32 SIMT kernels,
+ *     default options); pf_last_launch_count() and the profile list describe it like any other call.
+ *   - A problem whose scratch (pf_static_scratch_need(...) bytes: T', W, Uh and P of every chunk in fp32) exceeds
  *     PF_STATIC_SCRATCH_BYTES is refused with PF_ERR_WORKSPACE and nothing is launched.
  *   - The array occupies PF_STATIC_SCRATCH_BYTES on every GPU that loads the library, until exit.
  *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
@@ -147,6 +154,8 @@ int pf_deltanet_fwd_f32_static(const float* q, const float* k, const float* v, c
                                float* O, float* S_final, void* stream);
 /* The compiled-in value of PF_STATIC_SCRATCH_BYTES. */
 size_t pf_static_scratch_bytes(void);
+/* Bytes of the fixed array that pf_deltanet_fwd_f32_static would use for this problem (host arithmetic). */
+size_t pf_static_scratch_need(int B, int H, int L, int d_k, int d_v, int r, int chunk);
 
 typedef struct pf_params {
     const void* q;            /* as in pf_deltanet_fwd, element type given by in_dtype */
@@ -165,6 +174,26 @@ typedef struct pf_params {
     void* stream;
     int mode;                 /* PF_MODE_SUM (0) or PF_MODE_PRODUCT; anything else: PF_ERR_INVALID */
     int step;                 /* PF_STEP_EULER (0) or PF_STEP_EXACT; anything else: PF_ERR_INVALID */
+    /* Options.  0 always means the default; results agree within rounding whatever their values. */
+    int segments;             /* S > 1 (up to 64): cut every sequence into S segments of L/S tokens and evaluate them
+                                 side by side (Section 3, "Scan": the flow of an interval is the pair (P, Xi) with
+                                 S_end = S_start P + Xi, Proposition 2.1, and flows of consecutive intervals compose).
+                                 Three passes over the segments -- from the zero state (gives Xi), from the identity
+                                 (gives P + Xi), then, after a small kernel has composed the S flows of every sequence
+                                 into the segments' start states, from the true start states (gives O) -- so about three
+                                 times the work, but S times the parallelism: meant for problems with far fewer sequences
+                                 (B*H) than the GPU has SMs.  Needs d_k = d_v and L a multiple of S, otherwise
+                                 PF_ERR_UNSUPPORTED; the workspace grows by four arrays of B*H*S*d_k*d_v floats. */
+    int wu_builder;           /* how the fp32 SIMT kernels obtain W and Uh of a chunk.  0: the triangular inverse T' of
+                                 Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
+                                 "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one
+                                 kernel; needs more workspace.  The tensor-core kernels do not use it, except
+                                 PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels. */
+    int ring_depth;           /* 3..64 (default 8): slots per sequence of the L2-resident ring through which the
+                                 single-launch tensor-core path hands each chunk's flow to the state scan. */
+    int* status;              /* NULL, or a 4-byte aligned DEVICE word (owned by the caller) that receives the code of the
+                                 first bounded device-side wait that expired during this call (0 = none): see
+                                 pf_read_status. */
 } pf_params;
 
 /* Same operation with explicit options.  The workspace holds per-chunk intermediates (T', W, Uh, P
@@ -173,36 +202,46 @@ typedef struct pf_params {
  * named at PF_MODE_* and PF_STEP_*. */
 int pf_deltanet_fwd_ex(const pf_params* p);
 
-/* Bytes of scratch pf_deltanet_fwd_ex needs for this problem with this in_dtype/impl (0 on an
- * unsupported combination).  Host arithmetic; for the tensor-core implementations it asks the current
- * device for its SM count (no allocation, no launch, no synchronisation). */
+/* Bytes of scratch pf_deltanet_fwd_ex needs for this problem with this in_dtype/impl and every option at its
+ * default (0 on an unsupported combination).  Host arithmetic; for the tensor-core implementations it asks the
+ * current device for its SM count (no allocation, no launch, no synchronisation). */
 size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
+/* The same for a filled-in pf_params (shape, in_dtype, impl, mode and the options are read; pointers are not). */
+size_t pf_workspace_bytes_ex(const pf_params* p);
 
 /* Which PF_IMPL_* pf_deltanet_fwd_ex would run for this problem (negative pf_status if none). */
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
+/* The chunk length the kernels would be run with: `chunk` itself for an explicit implementation; under PF_IMPL_AUTO
+ * possibly another supported length (see PF_IMPL_AUTO).  Negative pf_status if the problem is not supported. */
+int pf_select_chunk(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl);
 
-/* Knobs (process-wide, not thread-safe; results agree within rounding whatever their values).  Returns PF_OK,
- * PF_ERR_UNSUPPORTED for an unknown name, PF_ERR_INVALID for a value out of range.
- *   "ring_depth" (3..64, default 8): slots per sequence of the L2-resident ring through which the
- *       single-launch tensor-core path hands each chunk's flow to the state scan.
- *   "flow_ctas" (0..1024, default 0 = no limit): upper limit on the CTAs of the single-launch path that build
- *       flows (the others scan); for measuring how the time scales with them.
- *   "wu_builder" (0 or 1, default 0): how the fp32 SIMT kernels obtain W and Uh of a chunk.  0: the triangular
- *       inverse T' of Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
- *       "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one kernel; it
- *       needs more workspace (pf_workspace_bytes follows the current value).  The tensor-core kernels do not
- *       use it, except PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels.
- *   "segments" (1..64, default 1): with S > 1 every forward call cuts each sequence into S segments of L/S
- *       tokens and evaluates them side by side (Section 3, "Scan": the flow of an interval is the pair (P, Xi)
- *       with S_end = S_start P + Xi, Proposition 2.1, and flows of consecutive intervals compose).  Three passes
- *       over the segments -- from the zero state (gives Xi), from the identity (gives P + Xi), then, after a
- *       small kernel has composed the S flows of every sequence into the segments' start states, from the true
- *       start states (gives O) -- so about three times the work, but S times the parallelism: meant for problems
- *       with far fewer sequences (B*H) than the GPU has SMs.  Needs d_k = d_v and L a multiple of S, otherwise
- *       the call returns PF_ERR_UNSUPPORTED (and pf_workspace_bytes 0); the workspace grows by four arrays of
- *       B*H*S*d_k*d_v floats.  A device-side timeout of an earlier pass is overwritten in the status word by
- *       the next pass on the tensor-core paths. */
-int pf_set_option(const char* name, int value);
+/*
+ * Device-side waits and the status word.
+ *
+ * The tensor-core kernels synchronise their warps, and the single-launch path its CTAs, with waits on barriers and
+ * flags.  Every such wait is bounded (about a second of SM cycles).  A wait that runs out writes its code into a
+ * 4-byte STATUS WORD and the kernels give up: they return, every other wait that sees the word set returns too, and
+ * O / S_final of that call are undefined.  Nothing traps, hangs or faults, and the context stays usable.
+ *
+ * Where the word lives, in this order: pf_params.status if given; else word 0 of pf_params.workspace if the caller
+ * passed one; else a word owned by the library (one per device).  Every forward call first sets the word it uses
+ * to 0, in stream order, so a word describes the LAST call that used it.
+ *
+ * pf_read_status(word, stream): synchronises `stream`, reads the word and returns PF_OK (0 in it) or PF_ERR_TIMEOUT.
+ * `word` is the pointer described above -- the status pointer, the workspace pointer, or NULL for the library's own
+ * word on the current device.  pf_last_wait_code() then gives the code that was read (host thread local):
+ *     1xx  flow-building role of the single-launch path (101-103 solve warps, 11x-12x bulk warps, 14x-15x MMA-issuing
+ *          warps, 16x flag warp),   2xx  its scanning role (20x chain, 21x output, 22x loads, 23x MMA issue),
+ *     1-99 the two-launch path (tc_flow, tc_scan),   99  shared memory not 1024-byte aligned,   900  pf_wait_selftest.
+ * The fp32 SIMT kernels have no such waits.
+ */
+int pf_read_status(const void* word, void* stream);
+int pf_last_wait_code(void);
+/* Diagnostic (no counterpart in the paper): launches one warp that waits, with the library's bounded-wait routine and a
+ * limit of `limit_us` microseconds (1..1000000), for a flag that nothing ever sets, so that the wait runs out, the
+ * status word (as for a forward call: `status`, or NULL for the library's own word) receives code 900 and the kernel
+ * returns.  For testing the reporting path above; it does not synchronise. */
+int pf_wait_selftest(int* status, int limit_us, void* stream);
 
 /* Number of kernels the last successful call on this host thread enqueued. */
 int pf_last_launch_count(void);

@@ -31,7 +31,8 @@ EXPORTS = [
     "pf_deltanet_fwd", "pf_deltanet_fwd_f32", "pf_deltanet_fwd_ex", "pf_workspace_bytes", "pf_select_impl",
     "pf_last_launch_count", "pf_status_string", "pf_last_error_string", "pf_version",
     "pf_profile_enable", "pf_profile_count", "pf_profile_read", "pf_tc_selftest",
-    "pf_deltanet_fwd_f32_static", "pf_static_scratch_bytes", "pf_set_option",
+    "pf_deltanet_fwd_f32_static", "pf_static_scratch_bytes", "pf_static_scratch_need",
+    "pf_workspace_bytes_ex", "pf_select_chunk", "pf_read_status", "pf_last_wait_code", "pf_wait_selftest",
 ]
 
 
@@ -47,6 +48,10 @@ class PfParams(ctypes.Structure):
         ("stream", ctypes.c_void_p),
         ("mode", ctypes.c_int),
         ("step", ctypes.c_int),
+        ("segments", ctypes.c_int),
+        ("wu_builder", ctypes.c_int),
+        ("ring_depth", ctypes.c_int),
+        ("status", ctypes.c_void_p),
     ]
 
 
@@ -97,8 +102,18 @@ def lib() -> ctypes.CDLL:
         L.pf_deltanet_fwd_f32_static.argtypes = [vp] * 5 + [ci] * 7 + [vp, vp, vp]
         L.pf_static_scratch_bytes.restype = ctypes.c_size_t
         L.pf_static_scratch_bytes.argtypes = []
-        L.pf_set_option.restype = ci
-        L.pf_set_option.argtypes = [ctypes.c_char_p, ci]
+        L.pf_static_scratch_need.restype = ctypes.c_size_t
+        L.pf_static_scratch_need.argtypes = [ci] * 7
+        L.pf_workspace_bytes_ex.restype = ctypes.c_size_t
+        L.pf_workspace_bytes_ex.argtypes = [ctypes.POINTER(PfParams)]
+        L.pf_select_chunk.restype = ci
+        L.pf_select_chunk.argtypes = [ci] * 9
+        L.pf_read_status.restype = ci
+        L.pf_read_status.argtypes = [vp, vp]
+        L.pf_last_wait_code.restype = ci
+        L.pf_last_wait_code.argtypes = []
+        L.pf_wait_selftest.restype = ci
+        L.pf_wait_selftest.argtypes = [vp, ci, vp]
         L.pf_tc_selftest.restype = ci
         L.pf_tc_selftest.argtypes = [ci, vp, vp, vp, ci, vp]
         _lib = L
@@ -188,11 +203,15 @@ def pf_static_scratch_bytes() -> int:
 
 
 def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Optional[torch.Tensor] = None,
-                       O=None, S_final=None, stream=None, want_state: bool = True, mode="sum", step="euler"):
+                       O=None, S_final=None, stream=None, want_state: bool = True, mode="sum", step="euler",
+                       segments: int = 0, wu_builder: int = 0, ring_depth: int = 0,
+                       status: Optional[torch.Tensor] = None):
     """Same operation with an explicit implementation and (optionally) a caller-owned workspace
-    (a uint8 CUDA tensor of at least pf_workspace_bytes(...) bytes).  mode: "sum" (the r factors of a token
+    (a uint8 CUDA tensor of at least pf_workspace_bytes_ex(...) bytes).  mode: "sum" (the r factors of a token
     read the same previous state) or "product" (they act one after another).  step: "euler" (the paper's
-    discretisation) or "exact" (each rank-1 factor takes exp(-beta k k^T); r = 1 or the product form)."""
+    discretisation) or "exact" (each rank-1 factor takes exp(-beta k k^T); r = 1 or the product form).
+    segments / wu_builder / ring_depth: the options of pf_params (0 = default).  status: an int32 CUDA tensor of one
+    element that receives the code of the first device-side wait that expired (see pf_read_status)."""
     dtype = q.dtype
     if dtype not in (torch.bfloat16, torch.float32):
         raise TypeError("q/k/v/beta must be bf16 or fp32")
@@ -209,11 +228,53 @@ def pf_deltanet_fwd_ex(q, k, v, beta, S0, chunk: int, impl="auto", workspace: Op
     p.stream = _stream(stream)
     p.mode = MODE_BY_NAME[mode] if isinstance(mode, str) else int(mode)
     p.step = STEP_BY_NAME[step] if isinstance(step, str) else int(step)
+    p.segments, p.wu_builder, p.ring_depth = int(segments), int(wu_builder), int(ring_depth)
+    if status is not None:
+        if status.dtype != torch.int32 or not status.is_cuda or status.numel() < 1:
+            raise ValueError("status must be an int32 CUDA tensor")
+        p.status = status.data_ptr()
     with torch.cuda.device(q.device):
         st = lib().pf_deltanet_fwd_ex(ctypes.byref(p))
     if st != 0:
         raise PfError(st, "pf_deltanet_fwd_ex")
     return O, S_final
+
+
+def pf_workspace_bytes_ex(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto", mode="sum", segments=0,
+                          wu_builder=0, ring_depth=0) -> int:
+    """pf_workspace_bytes with the options of pf_params taken into account."""
+    p = PfParams()
+    p.B, p.H, p.L, p.d_k, p.d_v, p.r, p.chunk = B, H, L, d_k, d_v, r, chunk
+    p.in_dtype = in_dtype
+    p.impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
+    p.mode = MODE_BY_NAME[mode] if isinstance(mode, str) else int(mode)
+    p.segments, p.wu_builder, p.ring_depth = int(segments), int(wu_builder), int(ring_depth)
+    return int(lib().pf_workspace_bytes_ex(ctypes.byref(p)))
+
+
+def pf_select_chunk(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
+    impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
+    return int(lib().pf_select_chunk(B, H, L, d_k, d_v, r, chunk, in_dtype, impl))
+
+
+def pf_read_status(word=None, stream=None) -> int:
+    """Synchronises the stream and returns 0 or -7 (PF_ERR_TIMEOUT).  `word`: the status tensor, the workspace tensor
+    (its word 0), or None for the library's own word on the current device."""
+    return int(lib().pf_read_status(None if word is None else word.data_ptr(), _stream(stream)))
+
+
+def pf_last_wait_code() -> int:
+    return int(lib().pf_last_wait_code())
+
+
+def pf_wait_selftest(status=None, limit_us: int = 1000, stream=None) -> None:
+    st = lib().pf_wait_selftest(None if status is None else status.data_ptr(), int(limit_us), _stream(stream))
+    if st != 0:
+        raise PfError(st, "pf_wait_selftest")
+
+
+def pf_static_scratch_need(B, H, L, d_k, d_v, r, chunk) -> int:
+    return int(lib().pf_static_scratch_need(B, H, L, d_k, d_v, r, chunk))
 
 
 def pf_workspace_bytes(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
@@ -224,12 +285,6 @@ def pf_workspace_bytes(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl
 def pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype=PF_DTYPE_BF16, impl="auto") -> int:
     impl = IMPL_BY_NAME[impl] if isinstance(impl, str) else int(impl)
     return int(lib().pf_select_impl(B, H, L, d_k, d_v, r, chunk, in_dtype, impl))
-
-
-def pf_set_option(name: str, value: int) -> None:
-    st = lib().pf_set_option(name.encode(), int(value))
-    if st != 0:
-        raise PfError(st, f"pf_set_option({name!r})")
 
 
 def pf_last_launch_count() -> int:

@@ -2,13 +2,17 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "pf_common.cuh"
 #include "pf_tc.cuh"
+#include "pf_tc_prims.cuh"
 
 namespace pf {
 
 static thread_local char g_err[512] = "";
 static thread_local int g_launches = 0;
+static thread_local int g_wait_code = 0;
 static thread_local int g_launch_accum = 0;
 
 int record_cuda_error(cudaError_t e, const char* where) {
@@ -47,6 +51,32 @@ void prof_end(cudaStream_t stream) {
 
 namespace {
 
+// The library's own status word (one per device that loads the library).  In host code the name is only a handle
+// for cudaGetSymbolAddress; its device address is looked up once per device.
+static __device__ int g_status_word;
+constexpr int kMaxDevices = 64;
+std::mutex g_status_mu;
+int* g_status_ptr[kMaxDevices] = {};
+
+int library_status_word(int** out) {
+    int dev = 0;
+    PF_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return PF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_status_mu);
+    if (!g_status_ptr[dev]) {
+        void* ptr = nullptr;
+        PF_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_status_word));
+        g_status_ptr[dev] = (int*)ptr;
+    }
+    *out = g_status_ptr[dev];
+    return PF_OK;
+}
+
+// One warp waits for a flag that nothing sets, with the bounded-wait routine of the kernels and a short limit.
+__global__ void wait_selftest_kernel(int* status, const int* flag, long long limit_cycles) {
+    if (threadIdx.x == 0) tc::flag_wait_ge_limit(flag, 1, status, 900, limit_cycles);
+}
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 int check_shape(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
@@ -57,21 +87,33 @@ int check_shape(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
     return PF_OK;
 }
 
-int g_wu_builder = 0;     // option "wu_builder"
-int g_segments = 1;       // option "segments"
-
 Problem as_problem(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype) {
     Problem p{};
     p.B = B; p.H = H; p.L = L; p.d_k = d_k; p.d_v = d_v; p.r = r; p.chunk = chunk;
     p.in_dtype = in_dtype;
-    p.wu_builder = g_wu_builder;
+    return p;
+}
+
+// option fields of pf_params: 0 = default
+int check_options(const pf_params* a) {
+    if (a->segments < 0 || a->segments > 64) return PF_ERR_INVALID;
+    if (a->wu_builder != 0 && a->wu_builder != 1) return PF_ERR_INVALID;
+    if (a->ring_depth != 0 && (a->ring_depth < 3 || a->ring_depth > 64)) return PF_ERR_INVALID;
+    if (a->status && ((uintptr_t)a->status & 3u)) return PF_ERR_ALIGNMENT;
+    return PF_OK;
+}
+Problem as_problem(const pf_params* a) {
+    Problem p = as_problem(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk, a->in_dtype);
+    p.mode = a->mode;
+    p.wu_builder = a->wu_builder;
+    p.ring_depth = a->ring_depth;
     return p;
 }
 
 // Picks the kernels.  The result of the operation does not depend on the chunk length (beyond rounding), so
 // PF_IMPL_AUTO may replace p.chunk by another supported length when that is what puts the problem on the tensor-core
-// kernels (they take 64 or 128 rows per chunk): config 3 with chunk 64 has 256 rows and would otherwise run on the
-// fp32 kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
+// kernels (they take 64 or 128 rows per chunk): r = 4 with chunk 64 has 256 rows and would otherwise run on the fp32
+// kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
 int select_impl(Problem& p, int impl) {
     if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
     p.auto_impl = impl == PF_IMPL_AUTO;
@@ -137,19 +179,20 @@ bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
     return a0 < b0 + bn && b0 < a0 + an;
 }
 
-// One forward call on the problem as given.  `top`: this is the caller's call itself (it resets and publishes the
-// launch count and the profile list); false for the passes of a segmented call.
-int forward_one(const pf_params* a, bool top) {
+}  // namespace
+
+// Checks that every entry point makes before anything is launched: shape, mode and step, pointers, alignment, O not
+// overlapping an input, device architecture.
+int check_call(const pf_params* a) {
     if (!a) return PF_ERR_INVALID;
     int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
     if (st != PF_OK) return st;
+    if (a->in_dtype != PF_DTYPE_BF16 && a->in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
     if (a->mode != PF_MODE_SUM && a->mode != PF_MODE_PRODUCT) return PF_ERR_INVALID;
     if (a->step != PF_STEP_EULER && a->step != PF_STEP_EXACT) return PF_ERR_INVALID;
     if (a->step == PF_STEP_EXACT && a->mode == PF_MODE_SUM && a->r != 1) return PF_ERR_UNSUPPORTED;   // rank-1 factors only
-    Problem p = as_problem(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk, a->in_dtype);
-    p.mode = a->mode;
-    const int impl = select_impl(p, a->impl);
-    if (impl < 0) return impl;
+    st = check_options(a);
+    if (st != PF_OK) return st;
     if (a->L > 0 && (!a->q || !a->k || !a->v || !a->beta || !a->O)) return PF_ERR_INVALID;
     if (!aligned16(a->q) || !aligned16(a->k) || !aligned16(a->v) || !aligned16(a->beta) || !aligned16(a->O) ||
         !aligned16(a->S0) || !aligned16(a->S_final))
@@ -160,12 +203,31 @@ int forward_one(const pf_params* a, bool top) {
     if (overlaps(a->O, o_bytes, a->q, th * a->d_k * es) || overlaps(a->O, o_bytes, a->k, th * a->r * a->d_k * es) ||
         overlaps(a->O, o_bytes, a->v, th * a->r * a->d_v * es) || overlaps(a->O, o_bytes, a->beta, th * a->r * es))
         return PF_ERR_INVALID;
-
     int dev = 0;
     PF_CUDA_TRY(cudaGetDevice(&dev));
     int major = 0;
     PF_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
     if (major != 10) return PF_ERR_ARCH;
+    return PF_OK;
+}
+
+// A new top-level call begins: the launch count and the profile list start over.
+void begin_call() {
+    g_launch_accum = 0;
+    g_prof_n = 0;
+}
+void end_call() { g_launches = g_launch_accum; }
+
+namespace {
+
+// One forward call on the problem as given.  `top`: this is the caller's call itself (it resets and publishes the
+// launch count and the profile list); false for the passes of a segmented call.
+int forward_one(const pf_params* a, bool top) {
+    int st = check_call(a);
+    if (st != PF_OK) return st;
+    Problem p = as_problem(a);
+    const int impl = select_impl(p, a->impl);
+    if (impl < 0) return impl;
 
     p.q = a->q; p.k = a->k; p.v = a->v; p.beta = a->beta; p.S0 = a->S0;
     p.O = a->O; p.S_final = a->S_final;
@@ -180,9 +242,23 @@ int forward_one(const pf_params* a, bool top) {
         PF_CUDA_TRY(cudaMallocAsync(&ws, need, p.stream));
         own = true;
     }
-    if (top) {
-        g_launch_accum = 0;
-        g_prof_n = 0;
+    if (top) begin_call();
+    // the status word of this call: the caller's, else word 0 of the caller's workspace, else the library's own
+    if (a->status) p.status = a->status;
+    else if (a->workspace) p.status = (int*)ws;
+    else {
+        st = library_status_word(&p.status);
+        if (st != PF_OK) {
+            if (own) cudaFreeAsync(ws, p.stream);
+            return st;
+        }
+    }
+    if (top) {      // (the passes of a segmented call share the word: the first expired wait of any of them stays)
+        cudaError_t e = cudaMemsetAsync(p.status, 0, sizeof(int), p.stream);
+        if (e != cudaSuccess) {
+            if (own) cudaFreeAsync(ws, p.stream);
+            return record_cuda_error(e, "cudaMemsetAsync(status)");
+        }
     }
     const long long rows = (long long)p.B * p.H * p.L * p.r;
     if (a->step == PF_STEP_EXACT && rows > 0) {
@@ -211,7 +287,7 @@ int forward_one(const pf_params* a, bool top) {
         cudaError_t e = cudaFreeAsync(ws, p.stream);
         if (e != cudaSuccess && st == PF_OK) st = record_cuda_error(e, "cudaFreeAsync");
     }
-    if (st == PF_OK && top) g_launches = g_launch_accum;
+    if (st == PF_OK && top) end_call();
     return st;
 }
 
@@ -297,22 +373,21 @@ pf_params seg_subproblem(const pf_params* a, int S) {
     pf_params b = *a;
     b.H = a->H * S;
     b.L = a->L / S;
+    b.segments = 0;
     return b;
 }
 size_t seg_workspace_need(const pf_params* a, int S) {
     const pf_params b = seg_subproblem(a, S);
-    Problem p = as_problem(b.B, b.H, b.L, b.d_k, b.d_v, b.r, b.chunk, b.in_dtype);
-    p.mode = b.mode;
+    Problem p = as_problem(&b);
     const int impl = select_impl(p, b.impl);
     if (impl < 0) return 0;
     return align_up(workspace_need(p, impl), 256) + 4 * seg_array_bytes(a, S);
 }
 
 int forward_segmented(const pf_params* a, int S) {
-    int st = check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk);
+    int st = check_call(a);
     if (st != PF_OK) return st;
     if (!seg_applicable(a, S)) return PF_ERR_UNSUPPORTED;
-    if (!aligned16(a->S0) || !aligned16(a->S_final)) return PF_ERR_ALIGNMENT;
     pf_params sub = seg_subproblem(a, S);
     const size_t need = seg_workspace_need(a, S);
     if (need == 0) return PF_ERR_UNSUPPORTED;
@@ -330,8 +405,26 @@ int forward_segmented(const pf_params* a, int S) {
     SegArrays arr{(float*)tail, (float*)(tail + ab), (float*)(tail + 2 * ab), (float*)(tail + 3 * ab)};
     sub.workspace = ws;
     sub.workspace_bytes = need - 4 * ab;
-    g_launch_accum = 0;
-    g_prof_n = 0;
+    begin_call();
+    // one status word for the three passes: the caller's, else word 0 of the workspace (as for an unsegmented call
+    // with a workspace), else the library's own; cleared once, so the first expired wait of any pass stays in it
+    if (!sub.status) {
+        if (a->workspace) sub.status = (int*)ws;
+        else {
+            st = library_status_word(&sub.status);
+            if (st != PF_OK) {
+                if (own) cudaFreeAsync(ws, stream);
+                return st;
+            }
+        }
+    }
+    {
+        cudaError_t e = cudaMemsetAsync(sub.status, 0, sizeof(int), stream);
+        if (e != cudaSuccess) {
+            if (own) cudaFreeAsync(ws, stream);
+            return record_cuda_error(e, "cudaMemsetAsync(status)");
+        }
+    }
     const int d = a->d_k;
     const long long slots = (long long)a->B * a->H * S;
     auto finish = [&](int code) {
@@ -376,13 +469,13 @@ int forward_segmented(const pf_params* a, int S) {
         cudaError_t e = cudaFreeAsync(ws, stream);
         if (e != cudaSuccess) return record_cuda_error(e, "cudaFreeAsync");
     }
-    g_launches = g_launch_accum;
+    end_call();
     return PF_OK;
 }
 
 int forward(const pf_params* a) {
     if (!a) return PF_ERR_INVALID;
-    if (g_segments > 1) return forward_segmented(a, g_segments);
+    if (a->segments > 1) return forward_segmented(a, a->segments);
     return forward_one(a, true);
 }
 
@@ -419,19 +512,22 @@ int pf_deltanet_fwd_f32(const float* q, const float* k, const float* v, const fl
     return pf::forward(&a);
 }
 
-size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
-    if (pf::check_shape(B, H, L, d_k, d_v, r, chunk) != PF_OK) return 0;
-    pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
-    const int sel = pf::select_impl(p, impl);
+size_t pf_workspace_bytes_ex(const pf_params* a) {
+    if (!a || pf::check_shape(a->B, a->H, a->L, a->d_k, a->d_v, a->r, a->chunk) != PF_OK || pf::check_options(a) != PF_OK) return 0;
+    if (a->mode != PF_MODE_SUM && a->mode != PF_MODE_PRODUCT) return 0;
+    if (a->segments > 1) return pf::seg_applicable(a, a->segments) ? pf::seg_workspace_need(a, a->segments) : 0;
+    pf::Problem p = pf::as_problem(a);
+    const int sel = pf::select_impl(p, a->impl);
     if (sel < 0) return 0;
-    if (pf::g_segments > 1) {
-        pf_params a;
-        memset(&a, 0, sizeof(a));
-        a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
-        a.in_dtype = in_dtype; a.impl = impl;
-        return pf::seg_applicable(&a, pf::g_segments) ? pf::seg_workspace_need(&a, pf::g_segments) : 0;
-    }
     return pf::workspace_need(p, sel);
+}
+
+size_t pf_workspace_bytes(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
+    pf_params a;
+    memset(&a, 0, sizeof(a));
+    a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
+    a.in_dtype = in_dtype; a.impl = impl;
+    return pf_workspace_bytes_ex(&a);
 }
 
 int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
@@ -441,22 +537,54 @@ int pf_select_impl(int B, int H, int L, int d_k, int d_v, int r, int chunk, int 
     return pf::select_impl(p, impl);
 }
 
-int pf_last_launch_count(void) { return pf::g_launches; }
-
-int pf_set_option(const char* name, int value) {
-    if (!name) return PF_ERR_INVALID;
-    if (strcmp(name, "segments") == 0) {
-        if (value < 1 || value > 64) return PF_ERR_INVALID;
-        pf::g_segments = value;
-        return PF_OK;
-    }
-    if (strcmp(name, "wu_builder") == 0) {
-        if (value != 0 && value != 1) return PF_ERR_INVALID;
-        pf::g_wu_builder = value;
-        return PF_OK;
-    }
-    return pf::fused_set_option(name, value);
+int pf_select_chunk(int B, int H, int L, int d_k, int d_v, int r, int chunk, int in_dtype, int impl) {
+    const int st = pf::check_shape(B, H, L, d_k, d_v, r, chunk);
+    if (st != PF_OK) return st;
+    pf::Problem p = pf::as_problem(B, H, L, d_k, d_v, r, chunk, in_dtype);
+    const int sel = pf::select_impl(p, impl);
+    return sel < 0 ? sel : p.chunk;
 }
+
+int pf_read_status(const void* word, void* stream) {
+    int* w = (int*)word;
+    if (!w) {
+        const int st = pf::library_status_word(&w);
+        if (st != PF_OK) return st;
+    }
+    int code = 0;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpy(&code, w, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return pf::record_cuda_error(e, "pf_read_status");
+    pf::g_wait_code = code;
+    return code == 0 ? PF_OK : PF_ERR_TIMEOUT;
+}
+
+int pf_last_wait_code(void) { return pf::g_wait_code; }
+
+int pf_wait_selftest(int* status, int limit_us, void* stream) {
+    if (limit_us < 1 || limit_us > 1000000) return PF_ERR_INVALID;
+    if (status && ((uintptr_t)status & 3u)) return PF_ERR_ALIGNMENT;
+    int* lib_word = nullptr;
+    int st = pf::library_status_word(&lib_word);
+    if (st != PF_OK) return st;
+    int* w = status ? status : lib_word;
+    int dev = 0, khz = 0;
+    PF_CUDA_TRY(cudaGetDevice(&dev));
+    PF_CUDA_TRY(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+    PF_CUDA_TRY(cudaMemsetAsync(w, 0, sizeof(int), (cudaStream_t)stream));
+    // the flag that nothing sets: a zeroed word in device memory, allocated on first use (this is a test helper)
+    static int* zero_flag[pf::kMaxDevices] = {};
+    if (!zero_flag[dev]) {
+        PF_CUDA_TRY(cudaMalloc((void**)&zero_flag[dev], 256));
+        PF_CUDA_TRY(cudaMemset(zero_flag[dev], 0, 256));
+    }
+    pf::wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(w, zero_flag[dev], (long long)limit_us * (khz / 1000));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return pf::record_cuda_error(e, "wait_selftest_kernel");
+    return PF_OK;
+}
+
+int pf_last_launch_count(void) { return pf::g_launches; }
 
 void pf_profile_enable(int on) { pf::g_prof_on = on != 0; }
 

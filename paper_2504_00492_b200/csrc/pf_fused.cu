@@ -1,4 +1,4 @@
-// fused: the whole tensor-core path in ONE cooperative launch (d_k = d_v = 128, n = C*r in {64, 128}).
+// fused: the whole tensor-core path in ONE cooperative launch (d_k = d_v = 128, chunks of n = C*r rows in tiles of 64 or 128).
 //
 // The paper's pipeline (Section 3) is Chunk -> Parallel Compute -> Scan.  Here both stages run at the same
 // time on disjoint sets of SMs and hand each chunk's flow over through a small ring that stays in L2:
@@ -18,33 +18,41 @@
 // rows of O that hold OI are updated by the scan a few chunk steps after the flow CTA wrote them, while they
 // are still in L2.  The only compulsory HBM traffic is one read of q, k, v, beta and one write of O.
 //
-// A flow CTA is software-pipelined over two chunks (15 warps, two teams of workers):
+// A flow CTA is software-pipelined over two chunks (16 warps):
 //   warps 0-3  "solve"  the chain that decides the period: epilogue of G = K K^T (mask, column scaling, fp16), the
-//                       16 x 16 diagonal blocks of the inverse (Neumann products on mma.sync, one warp per block)
-//                       and the recursive-doubling merges
+//                       16 x 16 diagonal blocks of the inverse (Neumann products (I-A)(I+A^2)(I+A^4)(I+A^8) on
+//                       mma.sync, two blocks per warp) and the recursive-doubling merges
 //   warps 4-11 "bulk"   one program for everything else, each step spread over all eight warps (two per lane
 //                       quarter of tensor memory): [Uh | W] into shared memory, P^T, bf16 -> fp16 of the next
-//                       chunk's V, K and Q, then the drains of E, Xi^T, Qt^T (into the ring) and OI (into O)
-//   warp 12             TMA loads (K and V double-buffered, Q single)
-//   warp 13             tcgen05.mma issue (whole warp, one elected lane per instruction)
+//                       chunk's V, K and Q in place, then the drains of E, Xi^T, Qt^T (into the ring) and OI (into
+//                       O); its first thread also issues the TMA loads (K and V double-buffered, Q single) at the
+//                       points of the program where their buffers fall free
+//   warps 12, 13, 15    tcgen05.mma issue, split by product so that no issuing warp waits behind another's operands:
+//                       13 polls (mbarrier.test_wait: try_wait may suspend the warp) for G of the next chunk and
+//                       [Uh | W] = X [V | K]; 12 issues E and Xi^T; 15 issues P0^T, Qt^T and OI^T
 //   warp 14             ring back-pressure and ready flags
 // Tensor memory: RA = columns [0,256) holds [Uh | W] and then [E | Xi^T]; RG = [256,384) holds G of the NEXT
 // chunk; RC = [384,448) holds P0^T and then Qt^T; RD = [448,512) holds OI^T.
 // G is formed from the bf16 tiles as they land (both operands raw); every other product has a derived fp16
-// operand, so K, V and Q are converted to fp16 in place, off the critical path.
+// operand, so K, V and Q are converted to fp16 in place, off the critical path.  Qt^T = Q^T - W^T P^T is formed
+// entirely on the tensor pipe: Q^T enters the accumulator as four products of the Q tile with a 16 x 16 identity,
+// then the correction accumulates onto it.
+// Every mbarrier is waited on by parity, so a waiter must never fall two phases behind its producer: the issue of
+// G for chunk k+1 is therefore gated on the bulk team having passed its own wait for G of chunk k.
 //
 // The images that cross the ring are laid out in unswizzled column groups (ns_off): a warp whose lanes hold
 // consecutive rows then writes 512 contiguous bytes per store, and the scan's bulk copies bring them into
 // shared memory in a form the MMA descriptors read directly.
 //
-// A scan CTA: warps 0-7 own the state (row j of S per thread, d_k split in two halves of 64 columns).  Each
-// chunk they write an fp16 copy of it into TENSOR memory, where it is the A operand of both of the chunk's
+// A scan CTA: warps 0-7 own the state in registers (row j of S per thread, d_k split in two halves of 64 columns).
+// Each chunk they write an fp16 copy of it into TENSOR memory, where it is the A operand of both of the chunk's
 // products (Delta = S E^T issued by warp 0, O^T = S Qt^T issued by warp 13), so the serial step never goes
 // through shared memory.  Warps 8-11 add OI and write O, warp 12 streams the E / Xi / Qt images in with bulk
 // copies and is the only poller of the ready flags, warp 14 reports consumed chunks.
 //
 // Every wait is bounded (about a second of cycles) and reports a code in the status word.  Outer loops are
-// deliberately kept rolled: the instruction footprint of fifteen differently-specialised warps matters.
+// deliberately kept rolled: the instruction footprint of sixteen differently-specialised warps matters.
+#include <atomic>
 #include <string.h>
 
 #include "pf_common.cuh"
@@ -892,22 +900,26 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t seqs, uint64_t rows, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (cached per device ordinal: a process may use several devices)
 int sm_count() {
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            sms = 0;
+    constexpr int MAX_DEV = 64;
+    static std::atomic<int> cache[MAX_DEV];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < MAX_DEV) {
+        const int have = cache[dev].load(std::memory_order_relaxed);
+        if (have) return have;
     }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < MAX_DEV) cache[dev].store(sms, std::memory_order_relaxed);
     return sms;
 }
 
-int g_ring_depth = 8;     // slots per sequence (option "ring_depth", 3..64)
-int g_flow_ctas = 0;      // upper limit on flow CTAs (option "flow_ctas"; 0 = every SM that is not scanning)
-
 int ring_depth(const Problem& p) {
+    const int want = p.ring_depth > 0 ? p.ring_depth : 8;     // slots per sequence (pf_params.ring_depth, 3..64)
     const int NC = p.chunks_per_seq();
-    return NC < g_ring_depth ? (NC < 1 ? 1 : NC) : g_ring_depth;
+    return NC < want ? (NC < 1 ? 1 : NC) : want;
 }
 
 struct Carve {
@@ -928,20 +940,6 @@ Carve carve(const Problem& p) {
 
 }  // namespace
 
-int fused_set_option(const char* name, int value) {
-    if (strcmp(name, "flow_ctas") == 0) {
-        if (value < 0 || value > 1024) return PF_ERR_INVALID;
-        g_flow_ctas = value;
-        return PF_OK;
-    }
-    if (strcmp(name, "ring_depth") == 0) {
-        if (value < 3 || value > 64) return PF_ERR_INVALID;
-        g_ring_depth = value;
-        return PF_OK;
-    }
-    return PF_ERR_UNSUPPORTED;
-}
-
 // One CTA per sequence scans, the rest build flows.  Measured at d = 128, r = 2: up to about 100 sequences the single
 // launch beats the two-launch form (96: 400 against 477 us at L = 2048), beyond that too few SMs are left for the
 // flows (120: 865 against 600 us; 136: 2194 against 669 us).
@@ -951,8 +949,7 @@ bool fused_preferred(const Problem& p) {
 
 bool fused_supported(const Problem& p) {
     if (p.in_dtype != PF_DTYPE_BF16 || p.d_k != DK || p.d_v != DV) return false;
-    const int n = p.n();
-    if (!(n == 64 || n == 128) || p.chunk > 64 || p.L < 1) return false;
+    if (p.tile_rows() == 0 || p.chunk > 64 || p.L < 1) return false;
     const long long nseq = (long long)p.B * p.H;
     const int sms = sm_count();
     if (sms < 16) return false;
@@ -969,7 +966,7 @@ int fused_forward(const Problem& p, void* workspace) {
     const Carve cv = carve(p);
     uint8_t* base = (uint8_t*)workspace;
     FusedWs ws;
-    ws.status = (int*)(base + cv.status);
+    ws.status = p.status;
     ws.ready = (int*)(base + cv.ready);
     ws.consumed = (int*)(base + cv.consumed);
     ws.ring = base + cv.ring;
@@ -980,14 +977,13 @@ int fused_forward(const Problem& p, void* workspace) {
     const int sms = sm_count();
     g.n_scan = nseq;
     g.n_flow = sms - nseq;
-    if (g_flow_ctas > 0 && g_flow_ctas < g.n_flow) g.n_flow = g_flow_ctas;
     if (g.items < g.n_flow) g.n_flow = g.items > 0 ? g.items : 1;
     FusedMaps maps;
     if (NC > 0) {
         const uint64_t seqs = (uint64_t)nseq;
-        if (!make_map(&maps.k, p.k, seqs, (uint64_t)p.L * p.r, p.d_k, p.n()) ||
+        if (!make_map(&maps.k, p.k, seqs, (uint64_t)p.L * p.r, p.d_k, p.tile_rows()) ||
             !make_map(&maps.q, p.q, seqs, (uint64_t)p.L, p.d_k, p.chunk) ||
-            !make_map(&maps.v, p.v, seqs, (uint64_t)p.L * p.r, p.d_v, p.n()))
+            !make_map(&maps.v, p.v, seqs, (uint64_t)p.L * p.r, p.d_v, p.tile_rows()))
             return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     } else {
         memset(&maps, 0, sizeof(maps));
@@ -997,7 +993,7 @@ int fused_forward(const Problem& p, void* workspace) {
     float* O = p.O;
     float* Sf = p.S_final;
     void* args[] = {(void*)&maps, (void*)&g, (void*)&ws, (void*)&beta, (void*)&S0, (void*)&O, (void*)&Sf};
-    const void* fn = p.n() == 128 ? (const void*)fused_kernel<128> : (const void*)fused_kernel<64>;
+    const void* fn = p.tile_rows() == 128 ? (const void*)fused_kernel<128> : (const void*)fused_kernel<64>;
     PF_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     prof_begin("fused", p.stream);
     PF_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3((unsigned)(g.n_scan + g.n_flow)), dim3(FT), args, SMEM_BYTES, p.stream));

@@ -46,18 +46,27 @@ int static_scratch(void** out) {
 
 extern "C" size_t pf_static_scratch_bytes(void) { return pf::kStaticScratchBytes; }
 
+extern "C" size_t pf_static_scratch_need(int B, int H, int L, int d_k, int d_v, int r, int chunk) {
+    pf::Problem p{};
+    p.B = B; p.H = H; p.L = L; p.d_k = d_k; p.d_v = d_v; p.r = r; p.chunk = chunk;
+    p.in_dtype = PF_DTYPE_F32;
+    return pf::simt_workspace_bytes(p);
+}
+
 extern "C" int pf_deltanet_fwd_f32_static(const float* q, const float* k, const float* v, const float* beta,
                                           const float* S0, int B, int H, int L, int d_k, int d_v, int r, int chunk,
                                           float* O, float* S_final, void* stream) {
     using namespace pf;
-    if (B < 1 || H < 1 || L < 0) return PF_ERR_INVALID;
-    if (!(d_k == 64 || d_k == 128) || !(d_v == 64 || d_v == 128) || r < 1 || r > 4 ||
-        !(chunk == 16 || chunk == 32 || chunk == 64))
-        return PF_ERR_UNSUPPORTED;
-    if (L > 0 && (!q || !k || !v || !beta || !O)) return PF_ERR_INVALID;
-    const uintptr_t any = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)beta | (uintptr_t)O |
-                          (uintptr_t)S0 | (uintptr_t)S_final;
-    if (any & 15u) return PF_ERR_ALIGNMENT;
+    // the same checks as the allocating entry point (shape, pointers, alignment, O not overlapping an input, device)
+    pf_params a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.S0 = S0;
+    a.B = B; a.H = H; a.L = L; a.d_k = d_k; a.d_v = d_v; a.r = r; a.chunk = chunk;
+    a.O = O; a.S_final = S_final;
+    a.in_dtype = PF_DTYPE_F32;
+    a.impl = PF_IMPL_SIMT;
+    a.stream = stream;
+    int st = check_call(&a);
+    if (st != PF_OK) return st;
 
     Problem p{};
     p.q = q; p.k = k; p.v = v; p.beta = beta; p.S0 = S0;
@@ -67,14 +76,13 @@ extern "C" int pf_deltanet_fwd_f32_static(const float* q, const float* k, const 
     p.stream = (cudaStream_t)stream;
     if (simt_workspace_bytes(p) > kStaticScratchBytes) return PF_ERR_WORKSPACE;   // too large for the fixed array
 
-    int dev = 0, major = 0;
-    PF_CUDA_TRY(cudaGetDevice(&dev));
-    PF_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
-    if (major != 10) return PF_ERR_ARCH;
     void* scratch = nullptr;
-    const int st = static_scratch(&scratch);
+    st = static_scratch(&scratch);
     if (st != PF_OK) return st;
     // Every word of the scratch that the kernels read is written earlier in the same call (gram writes
     // all of T and P, solve rewrites T, wu writes all of W and Uh), so nothing has to be cleared.
-    return simt_forward(p, scratch);
+    begin_call();
+    st = simt_forward(p, scratch);
+    if (st == PF_OK) end_call();
+    return st;
 }

@@ -295,7 +295,8 @@ size_t tc_ws_carve(const Problem& p, void* base, TcWs* out) {
     const size_t o_x = take(G * g.xi_bytes);
     if (out && base) {
         uint8_t* b = (uint8_t*)base;
-        out->err = (int*)(b + o_err);
+        out->err = p.status;     // (the first 1 KB of the workspace is reserved: its word 0 is the status word of callers that pass a workspace and no status pointer)
+        (void)o_err;
         out->E = b + o_e;
         out->Qt = b + o_q;
         out->Xi = b + o_x;
@@ -307,8 +308,7 @@ bool tc_scan_supported(const Problem& p) { return p.in_dtype == PF_DTYPE_BF16 &&
 
 bool tc_supported(const Problem& p) {
     if (!tc_scan_supported(p)) return false;
-    const int n = p.n();
-    if (!(n == 64 || n == 128)) return false;
+    if (p.tile_rows() == 0) return false;
     return tc_flow_available();
 }
 
@@ -342,7 +342,6 @@ int tc_forward_refflow(const Problem& p, void* workspace) {
     TcWs ws;
     const size_t tc_bytes = align_up(tc_ws_carve(p, workspace, &ws), 1024);
     void* simt_ws = (uint8_t*)workspace + tc_bytes;
-    PF_CUDA_TRY(cudaMemsetAsync(ws.err, 0, 1024, p.stream));
     float *Wf, *Uf, *Pf;
     int st = simt_prepare(p, simt_ws, &Wf, &Uf, &Pf);
     if (st != PF_OK) return st;
@@ -366,7 +365,6 @@ size_t tc_refflow_workspace_bytes(const Problem& p) {
 int tc_forward(const Problem& p, void* workspace) {
     TcWs ws;
     tc_ws_carve(p, workspace, &ws);
-    PF_CUDA_TRY(cudaMemsetAsync(ws.err, 0, 1024, p.stream));
     int st = tc_flow_launch(p, ws, pick_dvs(p));
     if (st != PF_OK) return st;
     return tc_scan_launch(p, ws);

@@ -36,7 +36,6 @@ bool fused_supported(const Problem& p);
 bool fused_preferred(const Problem& p);     // enough SMs are left for building flows that the single launch wins
 size_t fused_workspace_bytes(const Problem& p);
 int fused_forward(const Problem& p, void* workspace);
-int fused_set_option(const char* name, int value);
 
 // pf_simt.cu: runs the gram/solve/wu kernels only and returns where W, Uh and P were left.
 int simt_prepare(const Problem& p, void* workspace, float** W, float** U, float** P);

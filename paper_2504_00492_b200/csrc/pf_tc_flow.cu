@@ -112,16 +112,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     uint32_t tma_phase = 0, mma_phase = 0;
     bool ok = true;
-    // per-phase cycle counters of CTA 0 (diagnostic; words 32.. of the status block)
-    long long t_prev = clock64();
-    auto lap = [&](int phase) {
-        if (blockIdx.x == 0 && tid == 0) {
-            const long long now = clock64();
-            atomicAdd((unsigned long long*)(ws.err + 32) + phase, (unsigned long long)(now - t_prev));
-            t_prev = now;
-        }
-    };
-
     for (long long gc = blockIdx.x; gc < G && ok; gc += gridDim.x) {
         const long long seq = gc / g.NC;
         const int c = (int)(gc % g.NC);
@@ -150,8 +140,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         ok = mbar_wait(&tma_bar, tma_phase, err, 21);
         tma_phase ^= 1;
         if (!ok) break;
-
-        lap(0);
         // ---- bf16 -> fp16 in place (elementwise, so the swizzled layout is untouched) --------------------
         {
             constexpr int chunks = (SM::kq_bytes + SM::v_bytes) / 16;   // the two regions are contiguous
@@ -169,8 +157,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         fence_async_smem();
         __syncthreads();
-
-        lap(1);
         // ---- MMA1: [G | P0^T] = K [K;Q]^T ---------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -181,8 +167,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         mma_phase ^= 1;
         if (!ok) break;
         tc_fence_after();
-
-        lap(2);
         // ---- epilogue 1: A -> X buffer (fp16) + fp32 diagonal blocks; P^T -> fp16 -------------------------
         {
             const int tokm = m / r;
@@ -233,8 +217,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         tc_fence_before();
         __syncthreads();
-
-        lap(3);
         // ---- solve: 16x16 diagonal blocks by forward substitution (thread = one column of one block) ------
         if (tid < N) {
             const int b = tid >> 4, cc = tid & 15;
@@ -255,12 +237,9 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
                 *(__half*)(sX + slab_off(16 * b + mm, 16 * b + cc, N)) = __float2half_rn(x[mm]);
         }
         __syncthreads();
-        lap(4);
         merge_level<N, 16, 0>(x_b, sX, warp, lane);
         merge_level<N, 32, 0>(x_b, sX, warp, lane);
         if (N == 128) merge_level<N, 64, 0>(x_b, sX, warp, lane);
-
-        lap(5);
         // ---- T' = X diag(beta): the row owner scales its row by the column betas -----------------------------
         if (m < N) {
 #pragma unroll
@@ -277,8 +256,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         fence_async_smem();
         __syncthreads();
-
-        lap(6);
         // ---- MMA2: W = T' K,  Uh = T' V -------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -290,8 +267,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         mma_phase ^= 1;
         if (!ok) break;
         tc_fence_after();
-
-        lap(7);
         // 64 x 64 identity, fp16, slab layout, into the (now dead) X region: B operand of the "+ Q^T" product below
         for (int e = tid; e < 64 * 8; e += FLOW_THREADS) {
             const int row = e >> 3, ch = e & 7;
@@ -321,8 +296,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         fence_async_smem();
         tc_fence_before();
         __syncthreads();
-
-        lap(8);
         // ---- MMA3: E = -K^T W, Xi = K^T Uh;  MMA4: Qt^T = Q^T - W^T P^T, O_intra^T = Uh^T P^T ---------------
         if (tid == 0) {
             tc_fence_after();
@@ -337,8 +310,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         mma_phase ^= 1;
         if (!ok) break;
         tc_fence_after();
-
-        lap(9);
         // ---- epilogue 3: the chunk's flow -> workspace; O_intra -> O -----------------------------------
         {
             const int i = tid;   // accumulator lane: a d_k index (E, Xi, Qt^T) or a d_v index (O_intra^T)
@@ -398,7 +369,6 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
         }
         tc_fence_before();
         __syncthreads();   // shared and tensor memory are reused by the next chunk
-        lap(10);
     }
     tc_fence_before();
     __syncthreads();
@@ -460,7 +430,7 @@ bool tc_flow_available() { return true; }
 
 int tc_flow_launch(const Problem& p, const TcWs& ws, int dvs) {
     if (p.total_chunks() == 0) return PF_OK;
-    const int n = p.n();
+    const int n = p.tile_rows();       // box rows: the whole tile, rows past the chunk's own included (they get beta = 0)
     const uint64_t seqs = (uint64_t)p.B * p.H;
     FlowMaps maps;
     if (!make_map(&maps.k, p.k, seqs, (uint64_t)p.L * p.r, p.d_k, n) ||

@@ -133,18 +133,21 @@ __device__ __forceinline__ float ld_cg_f32(const float* p) {
     return v;
 }
 // Waits until *p >= want (acquire), bounded by elapsed cycles.
-static __device__ __noinline__ bool flag_wait_ge(const int* p, int want, int* err_flag, int code) {
+static __device__ __noinline__ bool flag_wait_ge_limit(const int* p, int want, int* err_flag, int code, long long limit) {
     if (ld_acquire_gpu(p) >= want) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (ld_acquire_gpu(p) >= want) return true;
         if ((it & 15u) == 0) {
-            if (clock64() - t0 > WAIT_CYCLES) break;
+            if (clock64() - t0 > limit) break;
             if ((it & 255u) == 0 && *(volatile int*)err_flag != 0) return false;
         }
     }
     atomicCAS(err_flag, 0, code);
     return false;
+}
+__device__ __forceinline__ bool flag_wait_ge(const int* p, int want, int* err_flag, int code) {
+    return flag_wait_ge_limit(p, want, err_flag, code, WAIT_CYCLES);
 }
 
 // Waits until a shared-memory counter reaches `want` (written by another warp of the CTA after

@@ -43,37 +43,33 @@ def test_config0_fp32():
     assert pf.pf_last_launch_count() > 0
 
 
+def _full_size_parity(w):
+    """One call of the plain entry point at full size against the oracle over every (b, h) sequence."""
+    import paper_2504_00492_b200 as pf
+    inp = pf_synth.make_inputs(w)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    assert pf.pf_read_status() == 0, pf.pf_last_wait_code()
+    assert torch.isfinite(O).all() and torch.isfinite(Sf).all()
+    O_ref, Sf_ref = util.run_oracle(inp)
+    O, Sf = O.cpu().numpy(), Sf.cpu().numpy()
+    eo, es = util.max_rel(O, O_ref), util.max_rel(Sf, Sf_ref)
+    print(f"{w.name}: max-normalised O {eo:.2e} S_final {es:.2e}; relative L2 O {util.rel_l2(O, O_ref):.2e} "
+          f"S_final {util.rel_l2(Sf, Sf_ref):.2e}")
+    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+    util.check_per_sequence(O, O_ref, util.TOL_BF16, w.name + " O")
+    util.check_per_sequence(Sf, Sf_ref, util.TOL_BF16, w.name + " S_final")
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c3_chunk32"])
 def test_full_configs(name):
     """Full benchmark sizes through the central call, in the configuration bench.py times."""
-    import paper_2504_00492_b200 as pf
-    w = pf_synth.CONFIGS[name]
-    inp = pf_synth.make_inputs(w)
-    d = inp.to("cuda")
-    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
-    torch.cuda.synchronize()
-    O_ref, Sf_ref = util.run_oracle(inp)
-    eo, es = util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
-    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
+    _full_size_parity(pf_synth.CONFIGS[name])
 
 
-def test_config4_long_context_sampled_heads():
-    """c4 at full size on the GPU; the oracle recomputes a sample of whole heads (heads are
-    independent sequences, so each sampled head is checked over all 65536 tokens)."""
-    import paper_2504_00492_b200 as pf
-    w = pf_synth.CONFIGS["c4"]
-    inp = pf_synth.make_inputs(w)
-    d = inp.to("cuda")
-    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
-    torch.cuda.synchronize()
-    heads = [0, 7, 18, 31]
-    sub = pf_synth.Inputs(inp.q[:, heads].contiguous(), inp.k[:, heads].contiguous(), inp.v[:, heads].contiguous(),
-                          inp.beta[:, heads].contiguous(), inp.S0[:, heads].contiguous())
-    O_ref, Sf_ref = util.run_oracle(sub)
-    eo = util.max_rel(O[:, heads].cpu().numpy(), O_ref)
-    es = util.max_rel(Sf[:, heads].cpu().numpy(), Sf_ref)
-    assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
-    assert torch.isfinite(O).all() and torch.isfinite(Sf).all()
+def test_long_context_all_heads():
+    """L = 65536 at full size; the oracle recomputes every one of the 32 heads over all tokens."""
+    _full_size_parity(pf_synth.CONFIGS["c4"])
 
 
 # --- properties that hold at any size -------------------------------------------------------------
@@ -176,24 +172,30 @@ TC_CASES = [
     Workload("tc_dk64_dv128", B=1, H=2, L=256, d_k=64, d_v=128, r=2, chunk=64, s0_std=0.1, seed=35),
     Workload("tc_dk128_dv64", B=1, H=2, L=256, d_k=128, d_v=64, r=2, chunk=32, s0_std=0.1, seed=36),
     Workload("tc_one_token", B=1, H=1, L=1, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=37),
+    # r = 3: 96 (48) rows per chunk in a tile of 128 (64), the rows past them switched off by beta = 0
+    Workload("tc_r3_d64_c32", B=2, H=2, L=333, d_k=64, d_v=64, r=3, chunk=32, beta_scale=2.0, s0_std=0.1, seed=48),
+    Workload("tc_r3_d64_c16", B=1, H=2, L=200, d_k=64, d_v=64, r=3, chunk=16, s0_std=0.1, seed=49),
+    Workload("tc_r3_dk64_dv128", B=1, H=2, L=256, d_k=64, d_v=128, r=3, chunk=32, s0_std=0.1, seed=50),
 ]
 
 
-def _run_with_status(w, impl, mode="sum", step="euler"):
+def _run_with_status(w, impl, mode="sum", step="euler", **options):
+    """Runs with a caller workspace, reads the device status word through pf_read_status, compares with the oracle."""
     import paper_2504_00492_b200 as pf
     from paper_2504_00492_b200 import binding
     inp = pf_synth.make_inputs(w)
     d = inp.to("cuda")
-    need = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, impl)
+    need = pf.pf_workspace_bytes_ex(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, impl, mode=mode,
+                                    **options)
     assert need > 0
     ws = torch.zeros(need + 256, dtype=torch.uint8, device="cuda")
     off = (-ws.data_ptr()) % 256
     O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl, workspace=ws[off:off + need],
-                                  mode=mode, step=step)
-    torch.cuda.synchronize()
-    status = int(ws[off:off + 4].view(torch.int32).item())
-    assert status == 0, f"device-side wait {status} expired"
+                                  mode=mode, step=step, **options)
+    st = pf.pf_read_status(ws[off:off + need])
+    assert st == 0, f"device-side wait {pf.pf_last_wait_code()} expired"
     O_ref, Sf_ref = util.run_oracle(inp, mode=mode, step=step)
+    util.check_per_sequence(O.cpu().numpy(), O_ref, util.TOL_BF16, w.name + " O")
     return util.max_rel(O.cpu().numpy(), O_ref), util.max_rel(Sf.cpu().numpy(), Sf_ref)
 
 
@@ -211,6 +213,39 @@ def test_tc_full_path(w):
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
 
 
+def _scaled(inp, factor):
+    return pf_synth.Inputs(inp.q, inp.k, inp.v * factor, inp.beta, None if inp.S0 is None else inp.S0 * factor)
+
+
+@pytest.mark.parametrize("impl", ["tc", "tc_split"])
+def test_values_near_the_top_of_the_documented_fp16_range(impl):
+    """v and S0 scaled by 2^10 (exact in bf16): the tensor-core paths hold them and the state in fp16, whose range the
+    header documents; the result is linear in (v, S0), so the normalised error must stay what it is unscaled."""
+    import paper_2504_00492_b200 as pf
+    w = Workload("range_1e3", B=1, H=2, L=512, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=38)
+    inp = _scaled(pf_synth.make_inputs(w), 1024.0)
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl=impl)
+    assert pf.pf_read_status() == 0
+    O_ref, Sf_ref = util.run_oracle(inp)
+    assert float(abs(O_ref).max()) > 100.0
+    assert torch.isfinite(O).all() and torch.isfinite(Sf).all()
+    assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16
+    assert util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
+
+
+def test_values_beyond_the_fp16_range_need_the_fp32_path():
+    """Scaled by 2^20 the fp16 operands overflow (documented); PF_IMPL_SIMT keeps fp32 throughout and still agrees."""
+    import paper_2504_00492_b200 as pf
+    w = Workload("range_1e6", B=1, H=1, L=256, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=39)
+    inp = _scaled(pf_synth.make_inputs(w), float(2 ** 20))
+    d = inp.to("cuda")
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt")
+    O_ref, Sf_ref = util.run_oracle(inp)
+    assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16
+    assert util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
+
+
 # --- single-launch tensor-core path (flow builders and state scan side by side) -----------------------
 
 FUSED_CASES = [
@@ -220,6 +255,8 @@ FUSED_CASES = [
     Workload("fu_r2_c32", B=1, H=3, L=450, d_k=128, d_v=128, r=2, chunk=32, seed=44),                   # n = 64, no S0
     Workload("fu_r4_c16", B=1, H=2, L=130, d_k=128, d_v=128, r=4, chunk=16, beta_scale=2.0, seed=45),   # n = 64, C = 16
     Workload("fu_short", B=3, H=1, L=17, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=46),         # less than a chunk
+    Workload("fu_r3_c32", B=2, H=2, L=1000, d_k=128, d_v=128, r=3, chunk=32, s0_std=0.1, seed=51),       # 96 rows in a tile of 128
+    Workload("fu_r3_c16", B=1, H=3, L=333, d_k=128, d_v=128, r=3, chunk=16, beta_scale=2.0, seed=52),   # 48 rows in a tile of 64
     Workload("fu_many_seq", B=5, H=28, L=192, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=47),    # 140 scan CTAs, 8 flow CTAs
 ]
 
@@ -237,15 +274,11 @@ def test_fused_and_split_agree_and_ring_depth_is_invisible():
     import paper_2504_00492_b200 as pf
     w = Workload("fu_vs_split", B=2, H=2, L=1500, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=48)
     d = pf_synth.make_inputs(w).to("cuda")
-    try:
-        outs = []
-        for depth in (3, 5, 8, 8, 21):
-            pf.pf_set_option("ring_depth", depth)
-            O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
-            torch.cuda.synchronize()
-            outs.append((O.clone(), Sf.clone()))
-    finally:
-        pf.pf_set_option("ring_depth", 8)
+    outs = []
+    for depth in (3, 5, 8, 0, 21):
+        O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc", ring_depth=depth)
+        assert pf.pf_read_status() == 0, pf.pf_last_wait_code()      # (no workspace, no status pointer: the library's word)
+        outs.append((O.clone(), Sf.clone()))
     for O, Sf in outs[1:]:
         assert torch.equal(O, outs[0][0]) and torch.equal(Sf, outs[0][1])
     O2, S2 = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc_split")
@@ -260,31 +293,45 @@ def test_too_many_sequences_take_the_two_launch_form():
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
 
 
-def test_set_option_rejects_bad_input():
+def test_options_reject_bad_values():
     import paper_2504_00492_b200 as pf
-    with pytest.raises(pf.PfError) as ei:
-        pf.pf_set_option("ring_depth", 2)
-    assert ei.value.status == -1
-    with pytest.raises(pf.PfError) as ei:
-        pf.pf_set_option("no_such_option", 1)
-    assert ei.value.status == -2
-    with pytest.raises(pf.PfError) as ei:
-        pf.pf_set_option("flow_ctas", -1)
-    assert ei.value.status == -1
-
-
-def test_flow_cta_limit_does_not_change_the_result():
-    import paper_2504_00492_b200 as pf
-    w = FUSED_CASES[0]
+    w = FUSED_CASES[5]
     d = pf_synth.make_inputs(w).to("cuda")
-    O0, S0_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
-    try:
-        for n in (1, 7, 40):
-            pf.pf_set_option("flow_ctas", n)
-            O1, S1_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc")
-            assert torch.equal(O0, O1) and torch.equal(S0_, S1_)
-    finally:
-        pf.pf_set_option("flow_ctas", 0)
+    for bad in (dict(ring_depth=2), dict(ring_depth=65), dict(wu_builder=2), dict(segments=-1), dict(segments=65)):
+        with pytest.raises(pf.PfError) as ei:
+            pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc", **bad)
+        assert ei.value.status == -1, bad
+        assert pf.pf_workspace_bytes_ex(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, impl="tc", **bad) == 0
+
+
+def test_an_expired_device_wait_is_reported():
+    """A wait that runs out: one warp waits (bounded, 200 us) for a flag that nothing sets.  The kernel returns, the
+    status word holds the code, pf_read_status reports PF_ERR_TIMEOUT, and the next forward call clears the word and
+    works -- nothing hangs or faults on the way."""
+    import paper_2504_00492_b200 as pf
+    for own in (False, True):
+        word = torch.zeros(1, dtype=torch.int32, device="cuda") if own else None
+        pf.pf_wait_selftest(word, limit_us=200)
+        assert pf.pf_read_status(word) == -7
+        assert pf.pf_last_wait_code() == 900
+        assert pf.pf_status_string(-7) == "device-side wait timed out"
+        w = FUSED_CASES[5]
+        inp = pf_synth.make_inputs(w)
+        d = inp.to("cuda")
+        O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="tc", status=word)
+        assert pf.pf_read_status(word) == 0 and pf.pf_last_wait_code() == 0
+        O_ref, Sf_ref = util.run_oracle(inp)
+        assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16
+        assert util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
+
+
+def test_chunk_length_that_auto_evaluates_with_is_reported():
+    import paper_2504_00492_b200 as pf
+    from paper_2504_00492_b200 import binding
+    assert pf.pf_select_chunk(8, 16, 4096, 64, 64, 4, 64) == 32                 # 256 rows per chunk: evaluated as chunk 32
+    assert pf.pf_select_chunk(8, 16, 4096, 64, 64, 4, 64, impl="simt") == 64    # explicit implementations keep it
+    assert pf.pf_select_chunk(2, 16, 8192, 128, 128, 2, 64) == 64
+    assert pf.pf_select_chunk(2, 16, 8192, 128, 128, 2, 48) == -2
 
 
 def test_back_to_back_launches_without_synchronisation():
@@ -397,53 +444,40 @@ def test_exact_step_changes_the_result_and_needs_rank_one_factors():
     assert e.value.status == -1
 
 
-# --- W and Uh from the two-index system of Theorem 3.3 (option "wu_builder" = 1) instead of the triangular inverse ----
-
-@pytest.fixture
-def wavefront_builder():
-    import paper_2504_00492_b200 as pf
-    pf.pf_set_option("wu_builder", 1)
-    yield
-    pf.pf_set_option("wu_builder", 0)
-
+# --- W and Uh from the two-index system of Theorem 3.3 (pf_params.wu_builder = 1) instead of the triangular inverse ----
 
 @pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_theorem_3_3_builder_simt(wavefront_builder, w, dtype):
-    util.check_parity(w.with_(dtype=dtype), impl="simt")
+def test_theorem_3_3_builder_simt(w, dtype):
+    util.check_parity(w.with_(dtype=dtype), impl="simt", wu_builder=1)
 
 
 @pytest.mark.parametrize("w", [SMALL[1], SMALL[3]], ids=lambda w: w.name)
-def test_theorem_3_3_builder_product_form_and_exact_step(wavefront_builder, w):
-    util.check_parity(w.with_(dtype="f32"), impl="simt", mode="product")
-    util.check_parity(w, impl="simt", mode="product", step="exact")
+def test_theorem_3_3_builder_product_form_and_exact_step(w):
+    util.check_parity(w.with_(dtype="f32"), impl="simt", mode="product", wu_builder=1)
+    util.check_parity(w, impl="simt", mode="product", step="exact", wu_builder=1)
 
 
-def test_theorem_3_3_builder_feeds_the_tensor_core_scan(wavefront_builder):
-    eo, es = _run_with_status(TC_CASES[0], "tc_refflow")
+def test_theorem_3_3_builder_feeds_the_tensor_core_scan():
+    eo, es = _run_with_status(TC_CASES[0], "tc_refflow", wu_builder=1)
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
 
 
-def test_the_two_builders_agree_closely_and_the_option_is_checked():
+def test_the_two_builders_agree_closely_and_need_different_workspaces():
     import paper_2504_00492_b200 as pf
     w = SMALL[3].with_(dtype="f32")
     d = pf_synth.make_inputs(w).to("cuda")
     O0, S0_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt")
     need0 = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt")
-    pf.pf_set_option("wu_builder", 1)
-    try:
-        O1, S1_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt")
-        need1 = pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt")
-        with pytest.raises(pf.PfError):
-            pf.pf_set_option("wu_builder", 2)
-    finally:
-        pf.pf_set_option("wu_builder", 0)
+    O1, S1_ = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, impl="simt", wu_builder=1)
+    need1 = pf.pf_workspace_bytes_ex(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt", wu_builder=1)
     assert need1 > need0
+    assert pf.pf_workspace_bytes(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, 1, "simt") == need0      # (no hidden state)
     assert util.max_rel(O1.cpu().numpy(), O0.cpu().numpy()) < 2 * util.TOL_F32
     assert util.max_rel(S1_.cpu().numpy(), S0_.cpu().numpy()) < 2 * util.TOL_F32
 
 
-# --- segments evaluated side by side, flows composed (option "segments") -----------------------------------------------
+# --- segments evaluated side by side, flows composed (pf_params.segments) -----------------------------------------------
 
 SEGMENT_CASES = [
     (Workload("sg_simt_f32", B=1, H=2, L=256, d_k=64, d_v=64, r=2, chunk=32, s0_std=0.1, seed=61, dtype="f32"), "simt", 4),
@@ -454,55 +488,46 @@ SEGMENT_CASES = [
 ]
 
 
-@pytest.fixture
-def segments():
-    import paper_2504_00492_b200 as pf
-
-    def set_(n):
-        pf.pf_set_option("segments", n)
-    yield set_
-    pf.pf_set_option("segments", 1)
-
-
 @pytest.mark.parametrize("w,impl,S", SEGMENT_CASES, ids=lambda x: getattr(x, "name", x))
-def test_segmented_evaluation(segments, w, impl, S):
-    segments(S)
+def test_segmented_evaluation(w, impl, S):
     if impl == "simt":
-        util.check_parity(w, impl=impl)
+        util.check_parity(w, impl=impl, segments=S)
     else:
-        eo, es = _run_with_status(w, impl)
+        eo, es = _run_with_status(w, impl, segments=S)
         assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
 
 
-def test_segmented_product_form_exact_step_and_plain_entry_point(segments):
+def test_segmented_product_form_exact_step_and_library_workspace():
     import paper_2504_00492_b200 as pf
-    segments(4)
     w = Workload("sg_modes", B=1, H=2, L=512, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=66)
-    eo, es = _run_with_status(w, "tc", mode="product", step="exact")
+    eo, es = _run_with_status(w, "tc", mode="product", step="exact", segments=4)
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
     inp = pf_synth.make_inputs(w)
     d = inp.to("cuda")
-    O, Sf = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)      # library-owned workspace
+    O, Sf = pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, segments=4)      # library-owned workspace
+    assert pf.pf_read_status() == 0
     O_ref, Sf_ref = util.run_oracle(inp)
     assert util.max_rel(O.cpu().numpy(), O_ref) <= util.TOL_BF16 and util.max_rel(Sf.cpu().numpy(), Sf_ref) <= util.TOL_BF16
+    # the plain entry points are not affected by anything an earlier call asked for
+    O2, _ = pf.pf_deltanet_fwd(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+    torch.cuda.synchronize()
+    assert pf.pf_last_launch_count() == 1
 
 
-def test_segments_that_do_not_fit_are_refused(segments):
+def test_segments_that_do_not_fit_are_refused():
     import paper_2504_00492_b200 as pf
-    segments(4)
     w = SMALL[0]                                   # d_k != d_v
     d = pf_synth.make_inputs(w).to("cuda")
     with pytest.raises(pf.PfError) as e:
-        pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+        pf.pf_deltanet_fwd_ex(d.q, d.k, d.v, d.beta, d.S0, w.chunk, segments=4)
     assert e.value.status == -2
     w2 = Workload("sg_bad_L", B=1, H=1, L=130, d_k=64, d_v=64, r=1, chunk=32, seed=67)     # 130 % 4 != 0
     d2 = pf_synth.make_inputs(w2).to("cuda")
     with pytest.raises(pf.PfError) as e:
-        pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk)
+        pf.pf_deltanet_fwd_ex(d2.q, d2.k, d2.v, d2.beta, d2.S0, w2.chunk, segments=4)
     assert e.value.status == -2
-    assert pf.pf_workspace_bytes(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, 0, "auto") == 0
-    with pytest.raises(pf.PfError):
-        pf.pf_set_option("segments", 0)
+    assert pf.pf_workspace_bytes_ex(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, 0, "auto", segments=4) == 0
+    assert pf.pf_workspace_bytes(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, 0, "auto") > 0
 
 
 # --- PF_IMPL_AUTO may evaluate with another chunk length to reach the tensor-core kernels ---------------------------------
@@ -510,7 +535,7 @@ def test_segments_that_do_not_fit_are_refused(segments):
 def test_auto_rechunks_onto_the_tensor_core_path():
     import paper_2504_00492_b200 as pf
     from paper_2504_00492_b200 import binding
-    # config 3's shape class: r = 4 with chunk 64 is 256 rows per chunk; chunk 32 gives the 128 the kernels take
+    # r = 4 with chunk 64 is 256 rows per chunk; chunk 32 gives the 128 the kernels take
     w = Workload("auto_r4_c64", B=2, H=2, L=500, d_k=64, d_v=64, r=4, chunk=64, beta_scale=2.0, s0_std=0.1, seed=71)
     assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
     assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "tc") == -2
@@ -521,9 +546,16 @@ def test_auto_rechunks_onto_the_tensor_core_path():
     w2 = Workload("auto_r1_c32", B=1, H=2, L=300, d_k=128, d_v=128, r=1, chunk=32, s0_std=0.1, seed=72)
     assert pf.pf_select_impl(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
     util.check_parity(w2, impl="auto")
-    # r = 3 never gives 64 or 128 rows: fp32 kernels, at the caller's chunk length
+    # r = 3 never gives 64 or 128 rows: its chunks sit in the next larger tile (48 rows in 64, 96 in 128); 192 rows
+    # do not fit, so chunk 64 is evaluated with a shorter chunk
     w3 = SMALL[2]
-    assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_SIMT
+    assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
+    assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "tc") == binding.PF_IMPL_TC
+    w4 = Workload("auto_r3_c64", B=2, H=2, L=700, d_k=128, d_v=128, r=3, chunk=64, s0_std=0.1, seed=73)
+    assert pf.pf_select_impl(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk, binding.PF_DTYPE_BF16, "tc") == -2
+    assert pf.pf_select_chunk(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk) in (32, 42)
+    util.check_parity(w4, impl="auto")
+    util.check_parity(w4.with_(d_k=64, d_v=64, name="auto_r3_c64_d64"), impl="auto")
 
 
 def test_auto_leaves_the_single_launch_when_few_sms_remain_for_flows():
