@@ -112,16 +112,17 @@ Problem as_problem(const pf_params* a) {
 
 // Picks the kernels.  The result of the operation does not depend on the chunk length (beyond rounding), so
 // PF_IMPL_AUTO may replace p.chunk by another supported length when that is what puts the problem on the tensor-core
-// kernels (they take 64 or 128 rows per chunk): r = 4 with chunk 64 has 256 rows and would otherwise run on the fp32
-// kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
+// kernels (they take up to 128 rows per chunk, in tiles of 64 or 128): r = 4 with chunk 64 has 256 rows and would
+// otherwise run on the fp32 kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
 int select_impl(Problem& p, int impl) {
     if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
     p.auto_impl = impl == PF_IMPL_AUTO;
     if (impl == PF_IMPL_AUTO && !tc_supported(p)) {
-        for (int c : {64, 32, 16}) {
+        // (42 tokens of r = 3 rows are 126 of a tile's 128 rows: the longest chunk of rank 3 that fits)
+        for (int c : {64, 42, 32, 16}) {
             Problem t = p;
             t.chunk = c;
-            if (tc_supported(t)) {
+            if ((c != 42 || (p.r == 3 && p.chunk > 42)) && tc_supported(t)) {
                 p.chunk = c;
                 break;
             }

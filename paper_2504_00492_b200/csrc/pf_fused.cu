@@ -241,8 +241,8 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
             // A = Mstrict (.) (G diag(beta)) as fp16 into X.  Warp w holds rows 32w .. 32w+31: the 32-column groups
-            // left of 32w lie entirely below the mask's edge, the group at 32w holds the edge, the groups to the
-            // right are zero.
+            // left of 32w lie entirely below the mask's edge (but for the last columns of the nearest one when the
+            // token groups of r = 3 rows straddle 32w), the group at 32w holds the edge, the groups to the right are zero.
             if (32 * warp < N) {
 #pragma unroll 1
                 for (int c0 = 0; c0 < N; c0 += 32) {
@@ -260,7 +260,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
                         bb[4 * j4] = bv.x; bb[4 * j4 + 1] = bv.y; bb[4 * j4 + 2] = bv.z; bb[4 * j4 + 3] = bv.w;
                     }
                     tmem_ld_wait();
-                    if (c0 < 32 * warp) {
+                    if (c0 + 32 <= ((32 * warp) / g.rm) * g.rm) {      // (below the edge for every row of the warp)
 #pragma unroll
                         for (int j8 = 0; j8 < 32; j8 += 8) {
                             float a[8];

@@ -553,7 +553,7 @@ def test_auto_rechunks_onto_the_tensor_core_path():
     assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "tc") == binding.PF_IMPL_TC
     w4 = Workload("auto_r3_c64", B=2, H=2, L=700, d_k=128, d_v=128, r=3, chunk=64, s0_std=0.1, seed=73)
     assert pf.pf_select_impl(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk, binding.PF_DTYPE_BF16, "tc") == -2
-    assert pf.pf_select_chunk(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk) in (32, 42)
+    assert pf.pf_select_chunk(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk) == 42         # 126 of a tile's 128 rows
     util.check_parity(w4, impl="auto")
     util.check_parity(w4.with_(d_k=64, d_v=64, name="auto_r3_c64_d64"), impl="auto")
 
