@@ -310,7 +310,7 @@ class SlicePipeline:
         self.first = False
 
 
-def kernel_profile(pf, d, w, steps):
+def kernel_profile(forward, d, steps):
     """Per-kernel device time (ms per launch, averaged) from CUDA events recorded inside the library."""
     from paper_2504_00492_b200 import binding
     lib = binding.lib()
@@ -320,14 +320,17 @@ def kernel_profile(pf, d, w, steps):
     lib.pf_profile_enable(1)
     acc = {}
     for _ in range(steps):
-        fwd_of(pf, w)(d.q, d.k, d.v, d.beta, d.S0, w.chunk)
+        forward(d.q, d.k, d.v, d.beta, d.S0)
         torch.cuda.synchronize()
         n = lib.pf_profile_count()
+        call = {}
         for i in range(n):
             name = ctypes.create_string_buffer(64)
             ms = ctypes.c_float(0)
             lib.pf_profile_read(i, name, 64, ctypes.byref(ms))
-            acc.setdefault(name.value.decode(), []).append(ms.value)
+            call[name.value.decode()] = call.get(name.value.decode(), 0.0) + ms.value     # (a kernel may run more than once per call)
+        for k, v in call.items():
+            acc.setdefault(k, []).append(v)
     lib.pf_profile_enable(0)
     return {k: statistics.mean(v) for k, v in acc.items()}
 
@@ -456,7 +459,7 @@ def main():
     e2e_launches = pf.pf_last_launch_count() * pipe.n
 
     # ---- per-kernel times and the roofline of the dominant kernel -----------------------------------------
-    prof = kernel_profile(pf, d, w, steps=min(args.steps, 5))
+    prof = kernel_profile(forward, d, steps=min(args.steps, 5))
     G = w.B * w.H * ((w.L + chunk_used - 1) // chunk_used)
     th = w.token_heads
     fl_tri = flops_per_chunk(w_eval, tri=True)

@@ -178,12 +178,15 @@ typedef struct pf_params {
     int segments;             /* S > 1 (up to 64): cut every sequence into S segments of L/S tokens and evaluate them
                                  side by side (Section 3, "Scan": the flow of an interval is the pair (P, Xi) with
                                  S_end = S_start P + Xi, Proposition 2.1, and flows of consecutive intervals compose).
-                                 Three passes over the segments -- from the zero state (gives Xi), from the identity
-                                 (gives P + Xi), then, after a small kernel has composed the S flows of every sequence
-                                 into the segments' start states, from the true start states (gives O) -- so about three
-                                 times the work, but S times the parallelism: meant for problems with far fewer sequences
-                                 (B*H) than the GPU has SMs.  Needs d_k = d_v and L a multiple of S, otherwise
-                                 PF_ERR_UNSUPPORTED; the workspace grows by four arrays of B*H*S*d_k*d_v floats. */
+                                 The pass is linear in (start state, v), so two passes over the segments suffice: from
+                                 the zero state with the caller's v (gives each segment's own part of O, and Xi) and from
+                                 the identity with v = 0 (gives P and, as its output, every token's response to its
+                                 segment's start state).  A small kernel composes the S flows of every sequence into the
+                                 segments' start states and one GEMM per segment adds start state x response to O.
+                                 About twice the work, but S times the parallelism and no pass waits for another's
+                                 states: meant for problems with far fewer sequences (B*H) than the GPU has SMs.  Needs
+                                 d_k = d_v and L a multiple of S, otherwise PF_ERR_UNSUPPORTED; the workspace grows by
+                                 four arrays of B*H*S*d_k*d_v floats, an O-sized array and a v-sized array of zeros. */
     int wu_builder;           /* how the fp32 SIMT kernels obtain W and Uh of a chunk.  0: the triangular inverse T' of
                                  Theorem 3.2, then W = T'K, Uh = T'V.  1: the two-index system of Theorem 3.3 (the
                                  "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one

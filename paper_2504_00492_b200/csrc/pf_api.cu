@@ -295,21 +295,32 @@ int forward_one(const pf_params* a, bool top) {
 // ---- segmented evaluation: the flows of S segments of every sequence in parallel, then their composition --------
 // Section 3, step 3 ("Scan"): the flow of an interval is the pair (P, Xi) with S_end = S_start P + Xi (Proposition 2.1),
 // and flows of consecutive intervals compose.  A sequence of L tokens is cut into S segments of L/S tokens, which the
-// kernels see as S independent sequences (the layout [B,H,L,...] makes that a change of H and L, not a copy):
-//   pass A: every segment from the zero state            -> S_final = Xi_seg
-//   pass B: every segment from the identity (d_v = d_k)  -> S_final = P_seg + Xi_seg   (row j of the state carries e_j P)
+// kernels see as S independent sequences (the layout [B,H,L,...] makes that a change of H and L, not a copy).  The
+// whole pass is linear in (S_start, v), so a segment's output splits into the part its own tokens write and the part
+// its start state contributes:
+//   pass A: every segment from the zero state, the caller's v   -> O_zero (into O),  S_final = Xi_seg
+//   pass R: every segment from the identity (d_v = d_k), v = 0  -> R[t][i] = (P_t q_t)[i], the query as the start state
+//           sees it (an O-shaped scratch),                         S_final = P_seg   (row j of the state carries e_j P)
 //   compose (one small kernel, serial over the S segments of a sequence, parallel over sequences and rows):
 //           start(0) = S0,  start(s+1) = start(s) P_s + Xi_s;  the last one is S_final
-//   pass C: every segment from its true start state      -> O
-// Three passes instead of one, but each is S times more parallel: worth it when B*H is far below the SM count.
+//   apply:  O[t][:] += start(s)^T-contracted R[t][:]   (one GEMM per segment, no serial dependence)
+// Two passes instead of one, each S times more parallel, and no pass waits for the composition: worth it when B*H is
+// far below the SM count.
 struct SegArrays {
     float* xi;      // [B*H*S][d_k][d_v]  pass A's S_final
-    float* pb;      // same, pass B's
-    float* start;   // same, start state of every segment (the S0 of pass C)
-    float* ident;   // same, identity in every slot (the S0 of pass B)
+    float* pb;      // same, pass R's
+    float* start;   // same, start state of every segment
+    float* ident;   // same, identity in every slot (the S0 of pass R)
 };
 size_t seg_array_bytes(const pf_params* a, int S) {
     return align_up((size_t)a->B * a->H * S * a->d_k * a->d_v * sizeof(float), 256);
+}
+size_t seg_response_bytes(const pf_params* a) {      // R: one fp32 d_k-vector per token-head
+    return align_up((size_t)a->B * a->H * a->L * a->d_k * sizeof(float), 256);
+}
+size_t seg_zero_v_bytes(const pf_params* a) {
+    const size_t es = a->in_dtype == PF_DTYPE_F32 ? 4 : 2;
+    return align_up((size_t)a->B * a->H * a->L * a->r * a->d_v * es, 256);
 }
 
 __global__ void seg_identity_kernel(float* __restrict__ out, long long slots, int d) {
@@ -319,21 +330,38 @@ __global__ void seg_identity_kernel(float* __restrict__ out, long long slots, in
     out[e] = r == c ? 1.f : 0.f;
 }
 
-// grid (B*H, d/16), 256 threads; thread (jj, ig): row j = 16*blockIdx.y + jj of the state, columns i = 8*ig .. 8*ig+7.
-// Arrays are in the API layout X[i][j] = S[j][i].
+// grid (B*H, d/16), 256 threads; thread (jj, tx): row j = 16*blockIdx.y + jj of the state, columns i = tx, tx + 16, ...
+// Arrays are in the API layout X[i][j] = S[j][i].  The steps are serial, so each step's P and Xi are fetched into
+// registers while the step before is being computed.
+template <int D>
 __global__ void __launch_bounds__(256) seg_compose_kernel(const float* __restrict__ S0, SegArrays arr,
-                                                          float* __restrict__ S_final, int S, int d) {
+                                                          float* __restrict__ S_final, int S) {
+    constexpr int d = D;
     extern __shared__ float sm[];
-    float* Ps = sm;                 // [d][d]   P[i'][i]
-    float* cur = sm + d * d;        // [16][d]  rows of the current state
+    constexpr int ld = d + 4;       // (padded: the threads of a warp read 16 consecutive rows of Ps, 16 bytes each, without bank conflicts)
+    float* Ps = sm;                 // [d][ld]  Ps[i][i'] = P[i'][i], as pass R's S_final stores it
+    float* cur = sm + d * ld;       // [16][d]  rows of the current state
     const long long bh = blockIdx.x;
     const int j0 = blockIdx.y * 16;
-    const int jj = threadIdx.x >> 4, ig = (threadIdx.x & 15) * (d / 16);
-    const int per = d / 16;         // columns per thread: 8 (d = 128) or 4 (d = 64)
+    const int jj = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    constexpr int per = d / 16;     // columns per thread: 8 (d = 128) or 4 (d = 64)
+    constexpr int NV = d * d / 4 / 256;     // 16-byte pieces of P per thread: 16 or 4
     for (int e = threadIdx.x; e < 16 * d; e += 256) {
         const int r = e / d, i = e % d;
         cur[e] = S0 ? S0[(bh * d + i) * d + j0 + r] : 0.f;
     }
+    float4 pv[NV];
+    float xv[per];
+    auto fetch = [&](int s) {
+        const long long slot = bh * S + s;
+        const float4* pb = (const float4*)(arr.pb + slot * d * d);
+        const float* xi = arr.xi + slot * d * d;
+#pragma unroll
+        for (int u = 0; u < NV; ++u) pv[u] = pb[u * 256 + threadIdx.x];
+#pragma unroll
+        for (int c = 0; c < per; ++c) xv[c] = xi[(long long)(tx + 16 * c) * d + j0 + jj];
+    };
+    fetch(0);
     __syncthreads();
     for (int s = 0; s < S; ++s) {
         const long long slot = bh * S + s;
@@ -342,22 +370,29 @@ __global__ void __launch_bounds__(256) seg_compose_kernel(const float* __restric
             const int r = e % 16, i = e / 16;
             st[(long long)i * d + j0 + r] = cur[r * d + i];
         }
-        const float* xi = arr.xi + slot * d * d;
-        const float* pb = arr.pb + slot * d * d;
-        // P[i'][i] = (P + Xi)[i'][i] - Xi[i'][i], both stored as [i][i']
-        for (int e = threadIdx.x; e < d * d; e += 256) {
-            const int i = e / d, ip = e % d;
-            Ps[ip * d + i] = pb[e] - xi[e];
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int e = (u * 256 + threadIdx.x) * 4;
+            *(float4*)(Ps + (e / d) * ld + (e % d)) = pv[u];
+        }
+        float acc[per];     // (indexed by unrolled loops only, so that it stays in registers)
+#pragma unroll
+        for (int c = 0; c < per; ++c) acc[c] = xv[c];
+        __syncthreads();
+        if (s + 1 < S) fetch(s + 1);
+        // (column i of the new row is a dot product along i', which is contiguous in both operands)
+#pragma unroll 2
+        for (int ip = 0; ip < d; ip += 4) {
+            const float4 a = *(const float4*)(cur + jj * d + ip);
+#pragma unroll
+            for (int c = 0; c < per; ++c) {
+                const float4 pq = *(const float4*)(Ps + (tx + 16 * c) * ld + ip);
+                acc[c] = fmaf(a.x, pq.x, fmaf(a.y, pq.y, fmaf(a.z, pq.z, fmaf(a.w, pq.w, acc[c]))));
+            }
         }
         __syncthreads();
-        float acc[8];
-        for (int c = 0; c < per; ++c) acc[c] = xi[(long long)(ig + c) * d + j0 + jj];
-        for (int ip = 0; ip < d; ++ip) {
-            const float a = cur[jj * d + ip];
-            for (int c = 0; c < per; ++c) acc[c] = fmaf(a, Ps[ip * d + ig + c], acc[c]);
-        }
-        __syncthreads();
-        for (int c = 0; c < per; ++c) cur[jj * d + ig + c] = acc[c];
+#pragma unroll
+        for (int c = 0; c < per; ++c) cur[jj * d + tx + 16 * c] = acc[c];
         __syncthreads();
     }
     if (S_final)
@@ -365,6 +400,123 @@ __global__ void __launch_bounds__(256) seg_compose_kernel(const float* __restric
             const int r = e % 16, i = e / 16;
             S_final[(bh * d + i) * d + j0 + r] = cur[r * d + i];
         }
+}
+
+// O[slot][t][j] += sum_i R[slot][t][i] start[slot][i][j]: grid (ceil(Lseg / 64), slots), 256 threads; a CTA takes 64
+// tokens of one segment, thread (ty, tx) the 4 tokens 4 ty .. 4 ty + 3 and the D/16 columns j = (D/16) tx ...
+template <int D>
+__global__ void __launch_bounds__(256) seg_apply_kernel(const float* __restrict__ R, const float* __restrict__ start,
+                                                        float* __restrict__ O, int Lseg) {
+    extern __shared__ float sm[];
+    float* Ss = sm;                 // [D][D]    start[i][j]
+    float* Rs = sm + D * D;         // [D][64]   R[t][i] transposed: the 4 tokens of a thread are one 16-byte load
+    constexpr int PER = D / 16;
+    const long long slot = blockIdx.y;
+    const int t0 = blockIdx.x * 64;
+    const float* st = start + slot * D * D;
+    for (int e = threadIdx.x; e < D * D / 4; e += 256) ((float4*)Ss)[e] = ((const float4*)st)[e];
+    const float* Rg = R + (slot * Lseg + t0) * (long long)D;
+    for (int e = threadIdx.x; e < 64 * D; e += 256) {
+        const int t = e / D, i = e % D;
+        Rs[i * 64 + t] = (t0 + t < Lseg) ? Rg[(long long)t * D + i] : 0.f;
+    }
+    __syncthreads();
+    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    float acc[4][PER];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < PER; ++c) acc[a][c] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < D; ++i) {
+        const float4 rv = *(const float4*)(Rs + i * 64 + 4 * ty);
+        float b[PER];
+#pragma unroll
+        for (int c4 = 0; c4 < PER / 4; ++c4) {
+            const float4 bv = *(const float4*)(Ss + i * D + PER * tx + 4 * c4);
+            b[4 * c4] = bv.x; b[4 * c4 + 1] = bv.y; b[4 * c4 + 2] = bv.z; b[4 * c4 + 3] = bv.w;
+        }
+#pragma unroll
+        for (int c = 0; c < PER; ++c) {
+            acc[0][c] = fmaf(rv.x, b[c], acc[0][c]);
+            acc[1][c] = fmaf(rv.y, b[c], acc[1][c]);
+            acc[2][c] = fmaf(rv.z, b[c], acc[2][c]);
+            acc[3][c] = fmaf(rv.w, b[c], acc[3][c]);
+        }
+    }
+    float* Og = O + (slot * Lseg + t0) * (long long)D;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int t = 4 * ty + a;
+        if (t0 + t >= Lseg) continue;
+        float4* row = (float4*)(Og + (long long)t * D + PER * tx);
+#pragma unroll
+        for (int c4 = 0; c4 < PER / 4; ++c4) {
+            float4 o = row[c4];
+            o.x += acc[a][4 * c4]; o.y += acc[a][4 * c4 + 1]; o.z += acc[a][4 * c4 + 2]; o.w += acc[a][4 * c4 + 3];
+            row[c4] = o;
+        }
+    }
+}
+
+// The same product with fp16 operands on mma.sync.m16n8k16 (fp32 accumulation), for the bf16 entry points, whose
+// kernels round the state and the queries to fp16 as well: grid (ceil(Lseg / 128), slots), 256 threads; warp w takes the
+// 16 tokens 16 w .. 16 w + 15 and all D columns.  Both operands sit in shared memory with their contraction index
+// contiguous and rows padded by 16 bytes, so that every fragment register is one conflict-free 32-bit load.
+template <int D>
+__global__ void __launch_bounds__(256) seg_apply_mma_kernel(const float* __restrict__ R, const float* __restrict__ start,
+                                                            float* __restrict__ O, int Lseg) {
+    extern __shared__ __align__(16) uint8_t smraw[];
+    constexpr int LD = D + 8;                       // halves per row
+    __half* As = (__half*)smraw;                    // [128 tokens][LD]   R[t][i]
+    __half* Bs = As + 128 * LD;                     // [D columns j][LD]  start[i][j] transposed
+    const long long slot = blockIdx.y;
+    const int t0 = blockIdx.x * 128;
+    const float* Rg = R + (slot * Lseg + t0) * (long long)D;
+    for (int e = threadIdx.x; e < 128 * D / 4; e += 256) {
+        const int t = e / (D / 4), i4 = (e % (D / 4)) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t0 + t < Lseg) v = *(const float4*)(Rg + (long long)t * D + i4);
+        *(uint2*)(As + t * LD + i4) = make_uint2(tc::pack_h2(v.x, v.y), tc::pack_h2(v.z, v.w));
+    }
+    const float* st = start + slot * D * D;
+    for (int e = threadIdx.x; e < D * D; e += 256) {
+        const int i = e / D, j = e % D;
+        Bs[j * LD + i] = __float2half_rn(st[e]);
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
+    float acc[D / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < D / 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    const __half* arow = As + (16 * warp + gid) * LD + 2 * tig;
+#pragma unroll
+    for (int k0 = 0; k0 < D; k0 += 16) {
+        uint32_t a[4];
+        a[0] = *(const uint32_t*)(arow + k0);
+        a[1] = *(const uint32_t*)(arow + 8 * LD + k0);
+        a[2] = *(const uint32_t*)(arow + k0 + 8);
+        a[3] = *(const uint32_t*)(arow + 8 * LD + k0 + 8);
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) {
+            const __half* brow = Bs + (8 * nt + gid) * LD + k0 + 2 * tig;
+            tc::mma_16816(acc[nt], a, *(const uint32_t*)brow, *(const uint32_t*)(brow + 8));
+        }
+    }
+    float* Og = O + (slot * Lseg + t0) * (long long)D;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int t = 16 * warp + gid + 8 * hh;
+        if (t0 + t >= Lseg) continue;
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) {
+            float2* o = (float2*)(Og + (long long)t * D + 8 * nt + 2 * tig);
+            float2 v = *o;
+            v.x += acc[nt][2 * hh];
+            v.y += acc[nt][2 * hh + 1];
+            *o = v;
+        }
+    }
 }
 
 bool seg_applicable(const pf_params* a, int S) {
@@ -377,12 +529,15 @@ pf_params seg_subproblem(const pf_params* a, int S) {
     b.segments = 0;
     return b;
 }
+size_t seg_tail_bytes(const pf_params* a, int S) {
+    return 4 * seg_array_bytes(a, S) + seg_response_bytes(a) + seg_zero_v_bytes(a);
+}
 size_t seg_workspace_need(const pf_params* a, int S) {
     const pf_params b = seg_subproblem(a, S);
     Problem p = as_problem(&b);
     const int impl = select_impl(p, b.impl);
     if (impl < 0) return 0;
-    return align_up(workspace_need(p, impl), 256) + 4 * seg_array_bytes(a, S);
+    return align_up(workspace_need(p, impl), 256) + seg_tail_bytes(a, S);
 }
 
 int forward_segmented(const pf_params* a, int S) {
@@ -402,13 +557,15 @@ int forward_segmented(const pf_params* a, int S) {
         own = true;
     }
     const size_t ab = seg_array_bytes(a, S);
-    uint8_t* tail = (uint8_t*)ws + (need - 4 * ab);
+    uint8_t* tail = (uint8_t*)ws + (need - seg_tail_bytes(a, S));
     SegArrays arr{(float*)tail, (float*)(tail + ab), (float*)(tail + 2 * ab), (float*)(tail + 3 * ab)};
+    float* resp = (float*)(tail + 4 * ab);
+    void* zero_v = (uint8_t*)resp + seg_response_bytes(a);
     sub.workspace = ws;
-    sub.workspace_bytes = need - 4 * ab;
+    sub.workspace_bytes = need - seg_tail_bytes(a, S);
     begin_call();
-    // one status word for the three passes: the caller's, else word 0 of the workspace (as for an unsegmented call
-    // with a workspace), else the library's own; cleared once, so the first expired wait of any pass stays in it
+    // one status word for both passes: the caller's, else word 0 of the workspace (as for an unsegmented call
+    // with a workspace), else the library's own; cleared once, so the first expired wait of either pass stays in it
     if (!sub.status) {
         if (a->workspace) sub.status = (int*)ws;
         else {
@@ -419,25 +576,23 @@ int forward_segmented(const pf_params* a, int S) {
             }
         }
     }
-    {
-        cudaError_t e = cudaMemsetAsync(sub.status, 0, sizeof(int), stream);
-        if (e != cudaSuccess) {
-            if (own) cudaFreeAsync(ws, stream);
-            return record_cuda_error(e, "cudaMemsetAsync(status)");
-        }
-    }
-    const int d = a->d_k;
-    const long long slots = (long long)a->B * a->H * S;
     auto finish = [&](int code) {
         if (own) cudaFreeAsync(ws, stream);
         return code;
     };
-    // pass A: zero start
+    {
+        cudaError_t e = cudaMemsetAsync(sub.status, 0, sizeof(int), stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(zero_v, 0, seg_zero_v_bytes(a), stream);
+        if (e != cudaSuccess) return finish(record_cuda_error(e, "cudaMemsetAsync(status, zero v)"));
+    }
+    const int d = a->d_k;
+    const long long slots = (long long)a->B * a->H * S;
+    // pass A: zero start, the caller's v
     sub.S0 = nullptr;
     sub.S_final = arr.xi;
     st = forward_one(&sub, false);
     if (st != PF_OK) return finish(st);
-    // pass B: identity start
+    // pass R: identity start, v = 0; its "output" is the response of every token to the start state
     {
         const long long total = slots * d * d;
         prof_begin("seg_identity", stream);
@@ -446,26 +601,51 @@ int forward_segmented(const pf_params* a, int S) {
         count_launch();
     }
     sub.S0 = arr.ident;
+    sub.v = zero_v;
+    sub.O = resp;
     sub.S_final = arr.pb;
     st = forward_one(&sub, false);
     if (st != PF_OK) return finish(st);
     // composition of the S flows of every sequence
     {
-        const int smem = (d * d + 16 * d) * (int)sizeof(float);
-        cudaError_t e = cudaFuncSetAttribute(seg_compose_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        const int smem = (d * (d + 4) + 16 * d) * (int)sizeof(float);
+        const void* fn = d == 128 ? (const void*)seg_compose_kernel<128> : (const void*)seg_compose_kernel<64>;
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_compose_kernel attribute"));
+        const float* s0 = a->S0;
+        float* sf = a->S_final;
+        int nseg = S;
+        void* args[] = {(void*)&s0, (void*)&arr, (void*)&sf, (void*)&nseg};
         prof_begin("seg_compose", stream);
-        seg_compose_kernel<<<dim3((unsigned)(a->B * a->H), (unsigned)(d / 16)), 256, smem, stream>>>(a->S0, arr, a->S_final, S, d);
+        e = cudaLaunchKernel(fn, dim3((unsigned)(a->B * a->H), (unsigned)(d / 16)), dim3(256), args, (size_t)smem, stream);
         prof_end(stream);
         count_launch();
-        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_compose_kernel"));
     }
-    // pass C: true start states
-    sub.S0 = arr.start;
-    sub.S_final = nullptr;
-    st = forward_one(&sub, false);
-    if (st != PF_OK) return finish(st);
+    // every segment's start state applied to its responses
+    {
+        const int Lseg = a->L / S;
+        const bool half_ops = a->in_dtype == PF_DTYPE_BF16;      // (the fp32 entry points keep fp32 throughout)
+        const int smem = half_ops ? (128 + d) * (d + 8) * 2 : (d * d + 64 * d) * (int)sizeof(float);
+        const void* fn = half_ops ? (d == 128 ? (const void*)seg_apply_mma_kernel<128> : (const void*)seg_apply_mma_kernel<64>)
+                                  : (d == 128 ? (const void*)seg_apply_kernel<128> : (const void*)seg_apply_kernel<64>);
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_apply_kernel attribute"));
+        const int rows = half_ops ? 128 : 64;
+        const dim3 grid((unsigned)((Lseg + rows - 1) / rows), (unsigned)slots);
+        const float* rp = resp;
+        const float* sp = arr.start;
+        float* op = a->O;
+        int lseg = Lseg;
+        void* args[] = {(void*)&rp, (void*)&sp, (void*)&op, (void*)&lseg};
+        prof_begin("seg_apply", stream);
+        e = cudaLaunchKernel(fn, grid, dim3(256), args, (size_t)smem, stream);
+        prof_end(stream);
+        count_launch();
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return finish(record_cuda_error(e, "seg_apply_kernel"));
+    }
     if (own) {
         cudaError_t e = cudaFreeAsync(ws, stream);
         if (e != cudaSuccess) return record_cuda_error(e, "cudaFreeAsync");
