@@ -84,10 +84,14 @@ enum { PF_STEP_EULER = 0, PF_STEP_EXACT = 1 };
 
 /* Which kernels evaluate the chunk form.
  *   PF_IMPL_AUTO : tensor-core path where it supports the shape/dtype, else the fp32 SIMT path.  The result does
- *                  not depend on the chunk length beyond rounding, so AUTO may evaluate with another supported
- *                  chunk length than the one passed when that puts the problem on the tensor-core kernels (64 or
- *                  128 rows per chunk: e.g. r = 4 with chunk 64 runs as chunk 32; pf_select_chunk tells which).  The
- *                  explicit choices below use `chunk` as given.
+ *                  not depend on the chunk length beyond rounding, so AUTO may evaluate with another chunk length
+ *                  than the one passed when that puts the problem on the tensor-core kernels, which take up to 128
+ *                  rows (chunk * r) per chunk: a chunk with more rows is evaluated as consecutive blocks of whole
+ *                  tokens (r = 4 with chunk 64 as blocks of 32 tokens, r = 3 with chunk 64 as blocks of 42), the
+ *                  block forward substitution of the chunk's triangular system with the coupling between blocks
+ *                  carried by the state; a chunk with fewer than 64 rows is lengthened.  pf_select_chunk tells which
+ *                  length is used.  PF_IMPL_TC and PF_IMPL_TC_SPLIT split long chunks into blocks the same way but
+ *                  never lengthen a chunk; PF_IMPL_SIMT and PF_IMPL_TC_REFFLOW use `chunk` as given.
  *   PF_IMPL_SIMT : fp32 FFMA kernels (any supported shape; the only path for PF_DTYPE_F32).
  *   PF_IMPL_TC   : tcgen05 tensor-core kernels (bf16 inputs); PF_ERR_UNSUPPORTED otherwise.  For
  *                  d_k = d_v = 128 with at most (SM count - 8) sequences this is ONE cooperative launch in

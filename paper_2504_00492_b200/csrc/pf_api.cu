@@ -110,16 +110,21 @@ Problem as_problem(const pf_params* a) {
     return p;
 }
 
-// Picks the kernels.  The result of the operation does not depend on the chunk length (beyond rounding), so
-// PF_IMPL_AUTO may replace p.chunk by another supported length when that is what puts the problem on the tensor-core
-// kernels (they take up to 128 rows per chunk, in tiles of 64 or 128): r = 4 with chunk 64 has 256 rows and would
-// otherwise run on the fp32 kernels, 30 times slower.  Explicit implementations use the caller's chunk length as given.
+// Picks the kernels.  The tensor-core kernels take up to 128 rows per chunk (tiles of 64 or 128).  A chunk with more
+// rows (r = 4 with chunk 64 has 256, r = 3 with chunk 64 has 192) is evaluated as consecutive blocks of whole tokens
+// with at most 128 rows each: block forward substitution of the chunk's triangular system (the block-triangular case
+// of the Proposition after Theorem 3.2), in which the coupling of a block to the blocks before it, A_21 [Uh_1 | W_1],
+// is carried by the state, because flows compose exactly (Proposition 2.1).  In effect p.chunk becomes the block
+// length; pf_select_chunk reports it.  PF_IMPL_AUTO also moves to a longer chunk when the caller's gives fewer than
+// 64 rows (the result does not depend on the chunk length beyond rounding); explicit implementations never lengthen it.
 int select_impl(Problem& p, int impl) {
     if (p.in_dtype != PF_DTYPE_BF16 && p.in_dtype != PF_DTYPE_F32) return PF_ERR_UNSUPPORTED;
     p.auto_impl = impl == PF_IMPL_AUTO;
-    if (impl == PF_IMPL_AUTO && !tc_supported(p)) {
-        // (42 tokens of r = 3 rows are 126 of a tile's 128 rows: the longest chunk of rank 3 that fits)
+    const bool tc_family = impl == PF_IMPL_AUTO || impl == PF_IMPL_TC || impl == PF_IMPL_TC_SPLIT;
+    if (tc_family && !tc_supported(p)) {
+        // (42 tokens of r = 3 rows are 126 of a tile's 128 rows: the longest block of rank 3 that fits)
         for (int c : {64, 42, 32, 16}) {
+            if (impl != PF_IMPL_AUTO && c >= p.chunk) continue;
             Problem t = p;
             t.chunk = c;
             if ((c != 42 || (p.r == 3 && p.chunk > 42)) && tc_supported(t)) {

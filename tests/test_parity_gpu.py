@@ -538,9 +538,14 @@ def test_auto_rechunks_onto_the_tensor_core_path():
     # r = 4 with chunk 64 is 256 rows per chunk; chunk 32 gives the 128 the kernels take
     w = Workload("auto_r4_c64", B=2, H=2, L=500, d_k=64, d_v=64, r=4, chunk=64, beta_scale=2.0, s0_std=0.1, seed=71)
     assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
-    assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "tc") == -2
+    # an explicit tensor-core choice splits the 256-row chunk into two blocks of 128 rows as well
+    assert pf.pf_select_impl(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, binding.PF_DTYPE_BF16, "tc") == binding.PF_IMPL_TC
+    assert pf.pf_select_chunk(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, impl="tc") == 32
     util.check_parity(w, impl="auto")
-    eo, es = _run_with_status(w, "auto")
+    for impl in ("auto", "tc", "tc_split"):
+        eo, es = _run_with_status(w, impl)
+        assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (impl, eo, es)
+    eo, es = _run_with_status(w.with_(d_k=128, d_v=128, name="tc_r4_c64_d128"), "tc")        # the single launch
     assert eo <= util.TOL_BF16 and es <= util.TOL_BF16, (eo, es)
     # r = 1 with chunk 32 is 32 rows: chunk 64 gives 64
     w2 = Workload("auto_r1_c32", B=1, H=2, L=300, d_k=128, d_v=128, r=1, chunk=32, s0_std=0.1, seed=72)
@@ -552,7 +557,9 @@ def test_auto_rechunks_onto_the_tensor_core_path():
     assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "auto") == binding.PF_IMPL_TC
     assert pf.pf_select_impl(w3.B, w3.H, w3.L, w3.d_k, w3.d_v, w3.r, w3.chunk, binding.PF_DTYPE_BF16, "tc") == binding.PF_IMPL_TC
     w4 = Workload("auto_r3_c64", B=2, H=2, L=700, d_k=128, d_v=128, r=3, chunk=64, s0_std=0.1, seed=73)
-    assert pf.pf_select_impl(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk, binding.PF_DTYPE_BF16, "tc") == -2
+    assert pf.pf_select_impl(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk, binding.PF_DTYPE_BF16, "tc") == binding.PF_IMPL_TC
+    # ... but an explicit choice never lengthens a chunk: r = 1 with chunk 32 (32 rows) stays outside the tensor-core set
+    assert pf.pf_select_impl(w2.B, w2.H, w2.L, w2.d_k, w2.d_v, w2.r, w2.chunk, binding.PF_DTYPE_BF16, "tc") == -2
     assert pf.pf_select_chunk(w4.B, w4.H, w4.L, w4.d_k, w4.d_v, w4.r, w4.chunk) == 42         # 126 of a tile's 128 rows
     util.check_parity(w4, impl="auto")
     util.check_parity(w4.with_(d_k=64, d_v=64, name="auto_r3_c64_d64"), impl="auto")
