@@ -196,8 +196,9 @@ typedef struct pf_params {
                                  "signature kernel inspired algorithm", no inverse), swept along its antidiagonals by one
                                  kernel; needs more workspace.  The tensor-core kernels do not use it, except
                                  PF_IMPL_TC_REFFLOW, whose flows come from the SIMT kernels. */
-    int ring_depth;           /* 3..64 (default 8): slots per sequence of the L2-resident ring through which the
-                                 single-launch tensor-core path hands each chunk's flow to the state scan. */
+    int ring_depth;           /* 3..64: slots per sequence of the L2-resident ring through which the single-launch
+                                 tensor-core path hands each chunk's flow to the state scan.  Default 8, and 16 for
+                                 sequences of more than 256 chunks while all rings together stay within 48 MB. */
     int* status;              /* NULL, or a 4-byte aligned DEVICE word (owned by the caller) that receives the code of the
                                  first bounded device-side wait that expired during this call (0 = none): see
                                  pf_read_status. */
