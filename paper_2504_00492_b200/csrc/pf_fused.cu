@@ -431,6 +431,14 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // ---- RA = [E | Xi^T]: h = 1: row m of E, h = 0: row m of Xi^T, one 16-byte piece per column group, into the ring
             if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
             tc_fence_after();
+            // ---- K of chunk k+2 into the buffer that the products of [E | Xi^T] of this chunk, the last to read it, are
+            //      done with (issued before the drain: the next Gram product but one waits for this tile)
+            if (bt == 0 && k + 2 < nk) {
+                int s2 = seq, c2 = c;
+                advance(s2, c2);
+                advance(s2, c2);
+                load_k(b, s2, c2);
+            }
             {
                 uint8_t* row = slot + (h ? SLOT_E : SLOT_XI) + m * 16;
                 const uint32_t src = RA + lane_base + (h ? 0 : DK);
@@ -449,13 +457,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
-            // ---- K of chunk k+2 into the buffer that [E | Xi^T] of this chunk has just finished reading
-            if (bt == 0 && k + 2 < nk) {
-                int s2 = seq, c2 = c;
-                advance(s2, c2);
-                advance(s2, c2);
-                load_k(b, s2, c2);
-            }
             // ---- h = 1: RC: Qt^T (row i = m of the Qt image);  h = 0: RD: OI^T[j][t] -> OI[t][j = m] (fp32) into the rows of O
             if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
             tc_fence_after();
