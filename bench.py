@@ -63,9 +63,13 @@ def flops_per_chunk(w, tri: bool) -> dict:
     }
 
 
-# DRAM bytes (read + write) of one launch of the single-launch kernel from an ncu capture, valid only for the
-# kernel sources it was taken on (their hash is stored with it): {workload: (sha256 of the sources, bytes)}.
-NCU_TRAFFIC = {"c2": ("63b2cbe9ed107556", 337494016 + 125681408)}
+# Figures from ncu captures of the single-launch kernel, valid only for the kernel sources they were taken on (the
+# hash of those sources is stored with them; the commands are in profiles/fused_kernel_c2.md):
+#   NCU_TRAFFIC      DRAM bytes (read + write) of one full-size launch: {workload: (hash, bytes)}
+#   NCU_TENSOR_PIPE  sm__pipe_tensor_cycles_active (% of peak, elapsed), captured on the half-size case
+#                    (--batch 1 --heads 16) under the section-capture size rule: {workload: (hash, percent, case)}
+NCU_TRAFFIC = {"c2": ("9e9cf8d9f808389c", 337141504 + 123692288)}
+NCU_TENSOR_PIPE = {"c2": ("9e9cf8d9f808389c", 17.47, "half-size case B=1 H=16 of c2")}
 
 
 def kernel_source_hash() -> str:
@@ -82,6 +86,13 @@ def ncu_traffic(w):
     if not ent or ent[0] != kernel_source_hash():
         return None        # no capture, or the kernel has changed since the counters were taken
     return ent[1]
+
+
+def ncu_tensor_pipe(w):
+    ent = NCU_TENSOR_PIPE.get(w.name)
+    if not ent or ent[0] != kernel_source_hash():
+        return None, None
+    return ent[1], ent[2]
 
 
 class ClockSampler:
@@ -320,6 +331,9 @@ def kernel_profile(forward, d, steps):
     lib.pf_profile_enable(1)
     acc = {}
     for _ in range(steps):
+        # two calls back to back, the second one read: its kernels start on a busy GPU, as in the timed region (the
+        # library's event list holds the latest call)
+        forward(d.q, d.k, d.v, d.beta, d.S0)
         forward(d.q, d.k, d.v, d.beta, d.S0)
         torch.cuda.synchronize()
         n = lib.pf_profile_count()
@@ -348,6 +362,9 @@ def main():
     ap.add_argument("--ring-depth", type=int, default=0, help="pf_params.ring_depth (0 = the library's default)")
     ap.add_argument("--segments", type=int, default=0, help="pf_params.segments (0 = the library's default)")
     ap.add_argument("--e2e-slices", type=int, default=8, help="(b,h) slices of the pipelined end-to-end run")
+    ap.add_argument("--path", default="auto", choices=["auto", "tc", "tc_split", "simt"],
+                    help="pf_params.impl: the kernels to run (auto = what the plain entry point does)")
+    ap.add_argument("--wu-builder", type=int, default=0, help="pf_params.wu_builder (fp32 SIMT kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = pf_synth.CONFIGS[args.workload]
@@ -372,10 +389,14 @@ def main():
         options["ring_depth"] = args.ring_depth
     if args.segments:
         options["segments"] = args.segments
+    if args.path != "auto":
+        options["impl"] = args.path
+    if args.wu_builder:
+        options["wu_builder"] = args.wu_builder
     in_dtype = pf.PF_DTYPE_F32 if w.dtype == "f32" else pf.PF_DTYPE_BF16
     # PF_IMPL_AUTO may evaluate with a shorter chunk than the one asked for (the recurrence's result does not depend
     # on it); the work counts below use the chunk length the kernels ran with.
-    chunk_used = pf.pf_select_chunk(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, in_dtype)
+    chunk_used = pf.pf_select_chunk(w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, in_dtype, args.path)
     w_eval = w.with_(chunk=chunk_used)
 
     def forward(q, k, v, beta, S0, O=None, S_final=None, stream=None):
@@ -459,7 +480,7 @@ def main():
     e2e_launches = pf.pf_last_launch_count() * pipe.n
 
     # ---- per-kernel times and the roofline of the dominant kernel -----------------------------------------
-    prof = kernel_profile(forward, d, steps=min(args.steps, 5))
+    prof = kernel_profile(forward, d, steps=min(args.steps, 10))
     G = w.B * w.H * ((w.L + chunk_used - 1) // chunk_used)
     th = w.token_heads
     fl_tri = flops_per_chunk(w_eval, tri=True)
@@ -490,7 +511,8 @@ def main():
                         "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(w), "ms_per_launch": prof[top],
                         "peaks": peak_kind, "bytes_per_launch": nbytes,
                         "tensor": {"tflops_dense": fl_d / (prof[top] * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
-                                   "frac": fl_d / (prof[top] * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+                                   "frac": fl_d / (prof[top] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                   "pipe_active_pct": ncu_tensor_pipe(w)[0], "pipe_active_from": ncu_tensor_pipe(w)[1]},
                         "kernel_ms": prof}
         else:
             steps_of = kernel_steps.get(top, list(fl_tri))
@@ -514,10 +536,10 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 in / f16 operands / f32 accumulate" if pf.pf_select_impl(
-                w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk) == pf.PF_IMPL_TC else "f32",
+                w.B, w.H, w.L, w.d_k, w.d_v, w.r, w.chunk, in_dtype, args.path) in (2, 4) else "f32",      # PF_IMPL_TC, PF_IMPL_TC_SPLIT
             "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d_k": w.d_k, "d_v": w.d_v, "r": w.r,
-                       "chunk": w.chunk, "chunk_evaluated": chunk_used, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
+                       "chunk": w.chunk, "chunk_evaluated": chunk_used, "path": args.path, "l2": "inputs+outputs (%.0f MB) larger than L2" % (
                            (host.nbytes() + O.numel() * 4) / 1e6), "parallelism": "replicas" if world > 1 else "1 GPU"},
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
             "token_heads_per_s": value * w.H,
