@@ -426,8 +426,6 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bar[B_PTREADY]);
-            // ---- conversions for chunk k+1 (while [E | Xi^T] of chunk k is formed)
-            if (k + 1 < nk && !convert_vk(k + 1)) return;
             // ---- RA = [E | Xi^T]: h = 1: row m of E, h = 0: row m of Xi^T, one 16-byte piece per column group, into the ring
             if (!PF_WAIT(B_SLOTOK, k & 1, 120) || !PF_WAIT(B_RADONE, k & 1, 124)) return;
             tc_fence_after();
@@ -457,6 +455,9 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             }
             tc_fence_before();
             mbar_arrive(&bar[B_RAFREE]);
+            // ---- conversions for chunk k+1: only now, so that they do not take shared-memory bandwidth from the products
+            //      of [E | Xi^T] (which hold the tensor-memory columns the next [Uh | W] waits for)
+            if (k + 1 < nk && !convert_vk(k + 1)) return;
             // ---- h = 1: RC: Qt^T (row i = m of the Qt image);  h = 0: RD: OI^T[j][t] -> OI[t][j = m] (fp32) into the rows of O
             if (!PF_WAIT(B_D4DONE, k & 1, 126)) return;
             tc_fence_after();
