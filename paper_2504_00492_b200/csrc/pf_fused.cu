@@ -37,8 +37,9 @@
 // operand, so K, V and Q are converted to fp16 in place, off the critical path.  Qt^T = Q^T - W^T P^T is formed
 // entirely on the tensor pipe: Q^T enters the accumulator as four products of the Q tile with a 16 x 16 identity,
 // then the correction accumulates onto it.
-// Every mbarrier is waited on by parity, so a waiter must never fall two phases behind its producer: the issue of
-// G for chunk k+1 is therefore gated on the bulk team having passed its own wait for G of chunk k.
+// Every mbarrier is waited on by parity, so a waiter must never fall two phases behind its producer: the bulk team
+// therefore waits for "G of chunk k complete" on a barrier of chunk k's K buffer, whose next phase cannot come before
+// the team itself has requested the tile of chunk k+2 into that buffer.
 //
 // The images that cross the ring are laid out in unswizzled column groups (ns_off): a warp whose lanes hold
 // consecutive rows then writes 512 contiguous bytes per store, and the scan's bulk copies bring them into
@@ -130,6 +131,7 @@ enum {
     B_D4DONE = 18,    // mma: [Qt^T | OI^T] complete (and everything issued before it)
     B_D4FREE = 19,    // bulk: RC (Qt^T) and RD (OI^T) drained
     B_RAFREE = 20,    // bulk: RA ([E | Xi^T]) drained
+    B_GK = 21,        // [2] mma: G complete, per K buffer (the bulk warps convert that K tile only then)
     B_OUTDONE = 27,   // bulk: the chunk's images are stored
     B_SLOTOK = 28,    // flag warp: the chunk's ring slot may be written
     B_RADONE = 29,    // mma: [E | Xi^T] complete
@@ -235,9 +237,11 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             // A failed wait must not strand the other threads at a named barrier: the first barrier after the
             // waits carries the outcome, and the whole warpgroup leaves together.
             bool ok = true;
-            // (G of chunk k is issued only once W of chunk k-2, in this X region, has been read by all of that chunk's products)
-            sB[m] = bm;     // (the beta half of chunk k-2 was last read by that chunk's [Uh | W] epilogue)
+            // (G of chunk k is issued only once W of chunk k-2, in this X region, has been read by all of that chunk's
+            //  products; by then the beta half of chunk k-2 has been read by that chunk's [Uh | W] epilogue as well, so it is
+            //  rewritten only after this wait: the solve warps may run far ahead of a bulk team that waits for a ring slot)
             ok = PF_WAIT(B_GDONE, k & 1, 102);
+            sB[m] = bm;
             tc_fence_after();
             if (!named_bar_and(1, 128, ok)) return;
             // A = Mstrict (.) (G diag(beta)) as fp16 into X.  Warp w holds rows 32w .. 32w+31: the 32-column groups
@@ -336,7 +340,7 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
             cvt_region(smem + bb * F_REGION + V_OFF, K_BYTES, bt, 256);
             fence_async_smem();
             mbar_arrive(&bar[B_V16 + bb]);
-            if (!PF_WAIT(B_KFULL + bb, ph, 111) || !PF_WAIT(B_GDONE, kk & 1, 110)) return false;
+            if (!PF_WAIT(B_KFULL + bb, ph, 111) || !PF_WAIT(B_GK + bb, ph, 110)) return false;
             cvt_region(smem + bb * F_REGION + K_OFF, K_BYTES, bt, 256);
             fence_async_smem();
             mbar_arrive(&bar[B_K16 + bb]);
@@ -521,16 +525,18 @@ __device__ void flow_role(const FusedMaps& maps, const FusedGeo& g, const FusedW
 #pragma unroll 1
         while (ip3 < nk) {
             bool progress = false;
-            // (G of chunk ig: its K tile has landed; the solve warps have drained G of chunk ig-1; the bulk warps have all seen
-            //  G of chunk ig-1 complete -- they convert that chunk's K only then -- so that nobody can miss a phase of the
-            //  barrier G completes on; and the last product of chunk ig-2 is done with W in the X region G's epilogue goes to)
-            if (ig < nk && mbar_test(&bar[B_KFULL + (ig & 1)], ph2(ig)) &&
-                (ig == 0 || (mbar_test(&bar[B_GFREE], (ig - 1) & 1) && mbar_test(&bar[B_K16 + ((ig - 1) & 1)], ph2(ig - 1)))) &&
+            // (G of chunk ig: its K tile has landed; the solve warps have drained G of chunk ig-1; and the last product of
+            //  chunk ig-2 is done with W in the X region G's epilogue goes to.  The bulk warps, which convert K of chunk ig
+            //  only after this product, wait for it on a barrier of that K buffer: its next phase is the Gram product of
+            //  chunk ig+2, whose tile they request themselves after that conversion, so they cannot miss a phase, and the
+            //  Gram product of the next chunk need not wait for them.)
+            if (ig < nk && mbar_test(&bar[B_KFULL + (ig & 1)], ph2(ig)) && (ig == 0 || mbar_test(&bar[B_GFREE], (ig - 1) & 1)) &&
                 (ig < 2 || mbar_test(&bar[B_D4DONE], (ig - 2) & 1))) {
                 tc_fence_after();
                 const uint32_t k_b = reg0 + (ig & 1) * F_REGION + K_OFF;
                 gemm_uni<false, false, N, DK, N, N, true>(RG, k_b, k_b);            // G = K K^T from the bf16 tile as it landed
                 commit_uni(&bar[B_GDONE]);
+                commit_uni(&bar[B_GK + (ig & 1)]);
                 ++ig;
                 progress = true;
             }
@@ -839,7 +845,7 @@ fused_kernel(const __grid_constant__ FusedMaps maps, FusedGeo g, FusedWs ws, con
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.v);
-            mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128);
+            mbar_init(&bar[B_GDONE], 1); mbar_init(&bar[B_GFREE], 128); mbar_init(&bar[B_GK], 1); mbar_init(&bar[B_GK + 1], 1);
             mbar_init(&bar[B_D2DONE], 1); mbar_init(&bar[B_WUREADY], 256);
             mbar_init(&bar[B_P0DONE], 1); mbar_init(&bar[B_PTREADY], 256);
             mbar_init(&bar[B_D4DONE], 1); mbar_init(&bar[B_RADONE], 1); mbar_init(&bar[B_D4FREE], 256); mbar_init(&bar[B_RAFREE], 256);
