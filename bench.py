@@ -68,8 +68,8 @@ def flops_per_chunk(w, tri: bool) -> dict:
 #   NCU_TRAFFIC      DRAM bytes (read + write) of one full-size launch: {workload: (hash, bytes)}
 #   NCU_TENSOR_PIPE  sm__pipe_tensor_cycles_active (% of peak, elapsed), captured on the half-size case
 #                    (--batch 1 --heads 16) under the section-capture size rule: {workload: (hash, percent, case)}
-NCU_TRAFFIC = {"c2": ("9e9cf8d9f808389c", 337141504 + 123692288)}
-NCU_TENSOR_PIPE = {"c2": ("9e9cf8d9f808389c", 17.47, "half-size case B=1 H=16 of c2")}
+NCU_TRAFFIC = {"c2": ("16732b90a2b7b496", 337161216 + 120871424)}
+NCU_TENSOR_PIPE = {"c2": ("16732b90a2b7b496", 15.99, "half-size case B=1 H=16 of c2")}
 
 
 def kernel_source_hash() -> str:
