@@ -36,11 +36,16 @@ namespace {
 constexpr int SCAN_STAGES = 3;
 constexpr int SCAN_THREADS = 256;
 
+// Dynamic shared memory of tc_scan (bytes from a 1024-aligned base), sized by d_k so that the d_k = 64 shapes fit two
+// CTAs per SM (64 KB each; at d_k = 128 it is 176 KB):
+//   SCAN_STAGES stages of [E image (d_k x d_k fp16) | Qt image (d_k x 64 fp16)], then two fp16 copies of the state
+//   slice (d_k rows of 128 bytes).
 struct ScanSmem {
-    // dynamic shared memory carve-up (bytes from a 1024-aligned base)
-    static constexpr int stage_bytes = 32768 + 16384;            // E (up to 128x128) + Qt (up to 128 x 64)
-    static constexpr int sb_off = SCAN_STAGES * stage_bytes;     // two S16 buffers of 16 KB
-    static constexpr int total = sb_off + 2 * 16384;
+    __host__ __device__ static int stage_bytes(int d_k) { return d_k * d_k * 2 + d_k * 128; }
+    __host__ __device__ static int qt_off(int d_k) { return d_k * d_k * 2; }
+    __host__ __device__ static int sb_off(int d_k) { return SCAN_STAGES * stage_bytes(d_k); }
+    __host__ __device__ static int sb_bytes(int d_k) { return d_k * 128; }
+    __host__ __device__ static int total(int d_k) { return sb_off(d_k) + 2 * sb_bytes(d_k); }
 };
 
 template <int DVS>
@@ -92,10 +97,10 @@ tc_scan(TcGeo g, TcWs ws, const float* __restrict__ S0, float* __restrict__ O, f
         if (NC > 0) load_xi(0);
         bool ok = true;
         for (int c = 0; c < NC && ok; ++c) {
-            uint8_t* sb = smem + ScanSmem::sb_off + (c & 1) * 16384;
-            // fp16 copy of the state as the B operand of both MMAs: row i, DVS columns
+            uint8_t* sb = smem + ScanSmem::sb_off(d_k) + (c & 1) * ScanSmem::sb_bytes(d_k);
+            // fp16 copy of the state as the B operand of both MMAs: row i, DVS columns (the buffer has d_k rows)
 #pragma unroll
-            for (int qd = 0; qd < DVS / 8; ++qd) {
+            for (int qd = 0; active && qd < DVS / 8; ++qd) {
                 uint4 pk;
                 pk.x = pack_h2(S[8 * qd + 0], S[8 * qd + 1]);
                 pk.y = pack_h2(S[8 * qd + 2], S[8 * qd + 3]);
@@ -169,10 +174,10 @@ tc_scan(TcGeo g, TcWs ws, const float* __restrict__ S0, float* __restrict__ O, f
                 if (c >= SCAN_STAGES) ok = mbar_wait(&empty_bar[s], ((c / SCAN_STAGES) - 1) & 1, err, 13);
                 if (ok) {
                     const size_t gc = (size_t)seq * NC + c;
-                    uint8_t* st = smem + s * ScanSmem::stage_bytes;
+                    uint8_t* st = smem + s * ScanSmem::stage_bytes(d_k);
                     mbar_expect_tx(&full_bar[s], e_bytes + q_bytes);
                     bulk_load(st, ws.E + gc * g.e_bytes, e_bytes, &full_bar[s]);
-                    bulk_load(st + 32768, ws.Qt + gc * g.q_bytes, q_bytes, &full_bar[s]);
+                    bulk_load(st + ScanSmem::qt_off(d_k), ws.Qt + gc * g.q_bytes, q_bytes, &full_bar[s]);
                 }
             }
             if (!__shfl_sync(0xffffffffu, ok, 0)) break;
@@ -186,9 +191,9 @@ tc_scan(TcGeo g, TcWs ws, const float* __restrict__ S0, float* __restrict__ O, f
                 ok = mbar_wait(&full_bar[s], (c / SCAN_STAGES) & 1, err, 14) && mbar_wait(&s_ready[b], (c >> 1) & 1, err, 15);
                 if (ok) {
                     tc_fence_after();
-                    const uint32_t e_base = smem_u32(smem + s * ScanSmem::stage_bytes);
-                    const uint32_t q_base = e_base + 32768;
-                    const uint32_t s_base = smem_u32(smem + ScanSmem::sb_off + b * 16384);
+                    const uint32_t e_base = smem_u32(smem + s * ScanSmem::stage_bytes(d_k));
+                    const uint32_t q_base = e_base + ScanSmem::qt_off(d_k);
+                    const uint32_t s_base = smem_u32(smem + ScanSmem::sb_off(d_k) + b * ScanSmem::sb_bytes(d_k));
                     // Delta^T[i, j] = sum_i' E[i, i'] S[j, i']
                     gemm_issue<false, true>(t_delta, e_base, d_k, s_base, 128, DVS, d_k, false, false);
                     mma_commit(&delta_done);
@@ -318,7 +323,7 @@ int tc_scan_launch(const Problem& p, const TcWs& ws) {
     const TcGeo g = tc_geo(p);
     const int dvs = pick_dvs(p);
     const long long nseq = (long long)p.B * p.H;
-    const int smem = ScanSmem::total + 1024;
+    const int smem = ScanSmem::total(p.d_k) + 1024;
     const unsigned grid = (unsigned)(nseq * (p.d_v / dvs));
     prof_begin("tc_scan", p.stream);
     if (dvs == 32) {
