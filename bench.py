@@ -217,7 +217,7 @@ class Ranks:
 
 
 def fwd_of(pf, w):
-    """The entry point for the workload's input type (config 0 is fp32, the others bf16)."""
+    """The entry point for the workload's input type (workload c0 is fp32, the others bf16)."""
     return pf.pf_deltanet_fwd_f32 if w.dtype == "f32" else pf.pf_deltanet_fwd
 
 
