@@ -62,6 +62,11 @@ struct FlowMaps {
     CUtensorMap q, k, v;
 };
 
+// Brings a tile into the L2 ahead of the load that will land it in shared memory (no completion to wait for).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int x, int y, int z) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
 
 template <int N, int DK, int DV>
 __global__ void __launch_bounds__(FLOW_THREADS, (FlowSmem<N, DK, DV>::two_per_sm ? 2 : 1))
@@ -129,6 +134,17 @@ tc_flow(const __grid_constant__ FlowMaps maps, TcGeo g, TcWs ws, const __nv_bflo
                 tma_load_3d(sKQ + h * SM::kq_rows * 128 + N * 128, &maps.q, 64 * h, t0, (int)seq, &tma_bar);
             }
             for (int h = 0; h < DV / 64; ++h) tma_load_3d(sV + h * N * 128, &maps.v, 64 * h, t0 * r, (int)seq, &tma_bar);
+            // the tiles of this CTA's next chunk into the L2: their load proper is issued only when this chunk is done
+            // with the buffers, and then finds them there
+            const long long gn = gc + gridDim.x;
+            if (gn < G) {
+                const int sn = (int)(gn / g.NC), tn = (int)(gn % g.NC) * C;
+                for (int h = 0; h < DK / 64; ++h) {
+                    tma_prefetch_3d(&maps.k, 64 * h, tn * r, sn);
+                    tma_prefetch_3d(&maps.q, 64 * h, tn, sn);
+                }
+                for (int h = 0; h < DV / 64; ++h) tma_prefetch_3d(&maps.v, 64 * h, tn * r, sn);
+            }
         }
         const int m = tid;
         float beta_m = 0.f;
