@@ -415,6 +415,8 @@ EXACT_CASES = [   # (workload, impl, mode): r = 1 in the sum form, any r in the 
     (FUSED_CASES[2], "tc", "sum"),
     (FUSED_CASES[0], "tc", "product"),
     (FUSED_CASES[1], "tc", "product"),
+    ([w for w in TC_CASES if w.name == "tc_r3_d64_c32"][0], "tc_split", "product"),      # rank 3: 96 rows in a tile of 128
+    ([w for w in FUSED_CASES if w.name == "fu_r3_c32"][0], "tc", "product"),
 ]
 
 
@@ -485,6 +487,7 @@ SEGMENT_CASES = [
     (Workload("sg_fused", B=1, H=2, L=2048, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=63), "tc", 8),
     (Workload("sg_fused_ragged", B=1, H=1, L=1000, d_k=128, d_v=128, r=2, chunk=64, s0_std=0.1, seed=64), "tc", 2),
     (Workload("sg_split_d64", B=1, H=2, L=512, d_k=64, d_v=64, r=4, chunk=32, beta_scale=2.0, seed=65), "tc_split", 4),
+    (Workload("sg_fused_r3", B=1, H=2, L=1536, d_k=128, d_v=128, r=3, chunk=64, s0_std=0.1, seed=68), "auto", 4),   # chunks of 42 tokens
 ]
 
 
